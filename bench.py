@@ -1,0 +1,393 @@
+#!/usr/bin/env python
+"""Benchmark of the fused low-rank router: routed tokens/s on B200 and fraction of its roofline.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c3] [--impl reference]
+
+One *step* is one pass of the whole hot path (z projection, logit tiles, running top-k, online log-sum-exp when
+the gate needs it, gates, expert histogram) over one synthetic batch of the workload, through the library's C
+interface.  Rank 0 prints ONE JSON line.  Under torchrun every rank routes its own batch (tokens are independent,
+no collective on the data path): weak scaling, value = tokens of all ranks / max-over-ranks device time.
+
+Timing: CUDA events on the launching stream, W warm-up steps, then exactly K timed steps bracketed by a barrier
+and a device synchronise.  Between steps the inputs are either larger than L2 or rotated over enough copies
+that the working set exceeds L2 (stated in ``config.l2``).
+
+``--impl reference`` times the CPU fp64 oracle (the deliberately slow, obviously-correct program the tests use),
+as it stands, on the host cores, on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+L2_BYTES = 126 * 1024 * 1024
+METRIC = "routed tokens/sec at 1 B200 and % of roofline (max of FLOP and HBM bound)"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=float(p["hbm_gbs"]), bf16_tflops=float(p["bf16_tflops"]),
+                    bf16_tflops_sustained=float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def algorithmic_work(T, h, r, M, k):
+    """FLOPs and bytes the method must do/move for one batch (the T x M logit matrix it avoids is not counted;
+    neither are the second MMA of the hi/lo split or L2 re-reads of R2)."""
+    flops = 2.0 * T * (h * r + r * M)
+    nbytes = 2.0 * T * h + 2.0 * h * r + 2.0 * r * M + 8.0 * T * k + 4.0 * M
+    return flops, nbytes
+
+
+def roofline(T, h, r, M, k, seconds, peaks, traffic=None):
+    flops, nbytes = algorithmic_work(T, h, r, M, k)
+    t_flop = flops / (peaks["bf16_tflops"] * 1e12)
+    t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+    if t_flop >= t_hbm:
+        ach = flops / seconds / 1e12
+        return dict(bound="tensor", achieved=ach, peak=peaks["bf16_tflops"], unit="TFLOP/s",
+                    frac=ach / peaks["bf16_tflops"], traffic=traffic, peak_source=peaks["source"] + " (burst)")
+    ach = nbytes / seconds / 1e9
+    return dict(bound="hbm", achieved=ach, peak=peaks["hbm_gbs"], unit="GB/s", frac=ach / peaks["hbm_gbs"],
+                traffic=traffic, peak_source=peaks["source"])
+
+
+# DRAM bytes per launch of route_tcgen05_kernel from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum);
+# the capture behind each figure is summarised under profiles/.  None = not captured for that workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index = index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        def pump():
+            for line in self.proc.stdout:
+                self.samples.append((time.time(), line.strip()))
+        self.thread = threading.Thread(target=pump, daemon=True)
+        self.thread.start()
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0, t1):
+        rows = [s for (t, s) in self.samples if t0 - 0.05 <= t <= t1 + 0.15] or [s for (_, s) in self.samples[-3:]]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+
+
+def describe(name, case, gate_mode):
+    return (f"{name}: T={case.T} h={case.h} r={case.r} M={case.M} k={case.k} "
+            f"gate={'full-softmax' if gate_mode else 'topk-softmax'} inputs={case.meta.get('dist')} seed={case.meta.get('seed')}")
+
+
+def oracle_rate(case, gate_mode, target_seconds=12.0):
+    """Tokens/s of the CPU oracle on a bounded prefix sample of the workload's tokens."""
+    import oracle
+    probe = min(case.T, 64)
+    t0 = time.perf_counter()
+    oracle.route(case.X[:probe], case.R1, case.R2, case.k, gate_mode)
+    dt = max(time.perf_counter() - t0, 1e-4)
+    n = int(min(case.T, max(probe, probe * target_seconds / dt)))
+    t0 = time.perf_counter()
+    oracle.route(case.X[:n], case.R1, case.R2, case.k, gate_mode)
+    dt = time.perf_counter() - t0
+    return n / dt, n, dt, oracle.threads()
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores, bounded sample per step."""
+    from paper_2609_36301_b200 import inputs
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    name = args.workload
+    gate_mode = inputs.CONFIGS[name]["gate_mode"] if args.gate_mode is None else args.gate_mode
+    full_T = inputs.CONFIGS[name]["T"]
+    case = inputs.make_config(name, gate_mode=gate_mode, T=min(full_T, 4096))
+    # size the per-step sample so that warmup+steps stay within ~2 minutes
+    probe = 32
+    t0 = time.perf_counter()
+    oracle.route(case.X[:probe], case.R1, case.R2, case.k, gate_mode)
+    per_tok = max(time.perf_counter() - t0, 1e-4) / probe
+    budget = 100.0 / max(1, args.steps + args.warmup)
+    n = int(max(8, min(case.T, budget / per_tok)))
+    for _ in range(args.warmup):
+        oracle.route(case.X[:n], case.R1, case.R2, case.k, gate_mode)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.route(case.X[:n], case.R1, case.R2, case.k, gate_mode)
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"first {n} tokens of the workload per step (of {full_T}); fp64 oracle, OpenMP over tokens"
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=dt / args.steps * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=describe(name, case, gate_mode).replace(f"T={case.T}", f"T={full_T}")),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.threads(), kind="oracle", sample=sample),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def time_router(mr, torch, bufs, k, gate_mode, steps, warmup, stream):
+    """bufs: list of (X, R1, R2, idx, gate, counts) rotated step by step.  Returns seconds for `steps` steps."""
+    n = len(bufs)
+    for i in range(warmup):
+        X, R1, R2, idx, gate, counts = bufs[i % n]
+        mr.more_route(X, R1, R2, k, gate_mode, idx, gate, counts, stream)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream.synchronize()
+    ev0.record(stream)
+    for i in range(steps):
+        X, R1, R2, idx, gate, counts = bufs[i % n]
+        mr.more_route(X, R1, R2, k, gate_mode, idx, gate, counts, stream)
+    ev1.record(stream)
+    stream.synchronize()
+    return ev0.elapsed_time(ev1) * 1e-3
+
+
+def make_bufs(torch, case, copies):
+    def dev(a):
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    X0, R1, R2 = dev(case.X), dev(case.R1), dev(case.R2)
+    bufs = []
+    for c in range(copies):
+        X = X0 if c == 0 else X0.clone()
+        bufs.append((X, R1 if c == 0 else R1.clone(), R2 if c == 0 else R2.clone(),
+                     torch.empty((case.T, case.k), dtype=torch.int32, device="cuda"),
+                     torch.empty((case.T, case.k), dtype=torch.float32, device="cuda"),
+                     torch.empty((case.M,), dtype=torch.int32, device="cuda")))
+    return bufs
+
+
+def copies_for(case):
+    x_bytes = case.T * case.h * 2
+    if x_bytes > 2 * L2_BYTES:
+        return 1, f"inputs larger than L2 (X is {x_bytes / 1e6:.0f} MB, L2 126 MB)"
+    c = int(np.ceil(3 * L2_BYTES / x_bytes))
+    return c, f"rotating over {c} copies of the inputs/outputs ({c * x_bytes / 1e6:.0f} MB of X > L2 126 MB)"
+
+
+def unfused_reference_ms(torch, bufs, case, gate_mode, iters=5):
+    """Context only: the unfused low-rank router built from library ops (two matmuls, logits in HBM, top-k)."""
+    X, R1, R2 = bufs[0][:3]
+    def step():
+        z = X @ R1
+        logits = (z @ R2).float()
+        top, idx = torch.topk(logits, case.k, dim=1)
+        if gate_mode == 0:
+            g = torch.softmax(top, dim=1)
+        else:
+            g = torch.exp(top - torch.logsumexp(logits, dim=1, keepdim=True))
+        c = torch.bincount(idx.reshape(-1), minlength=case.M)
+        return g, c
+    try:
+        for _ in range(2):
+            step()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(iters):
+            step()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / iters
+    except Exception:
+        return None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--workload", default="c3")
+    ap.add_argument("--gate-mode", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-others", action="store_true", help="skip the per-configuration table")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    from paper_2609_36301_b200 import binding as mr
+    from paper_2609_36301_b200 import inputs
+
+    mr.lib()                                           # fail loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl")
+    peaks = load_peaks()
+    name = args.workload
+    gate_mode = inputs.CONFIGS[name]["gate_mode"] if args.gate_mode is None else args.gate_mode
+    case = inputs.make_config(name, seed=rank, gate_mode=gate_mode)
+    copies, l2_note = copies_for(case)
+    bufs = make_bufs(torch, case, copies)
+    stream = torch.cuda.Stream()
+    k = case.k
+
+    # ---- device-resident timing: W warm-up, K timed steps, barrier + sync on both sides
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    time_router(mr, torch, bufs, k, gate_mode, 0, args.warmup, stream)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    l0 = mr.launches()
+    w0 = time.time()
+    secs = time_router(mr, torch, bufs, k, gate_mode, args.steps, 0, stream)
+    torch.cuda.synchronize()
+    w1 = time.time()
+    if dist:
+        dist.barrier()
+    launches = mr.launches() - l0
+    clocks = sampler.summary(w0, w1)
+    sampler.stop()
+    status = mr.more_route_status(stream)
+    if status != 0:
+        raise SystemExit(f"device status {status}: {mr.strerror(status)}")
+    if dist:
+        t = torch.tensor([secs], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        secs = float(t.item())
+    value = world * case.T * args.steps / secs
+
+    # ---- end to end through the host-buffer entry point (pinned host memory, copies inside the timed region)
+    Xh = torch.from_numpy(case.X.view(np.int16)).pin_memory()
+    R1h = torch.from_numpy(case.R1.view(np.int16)).pin_memory()
+    R2h = torch.from_numpy(case.R2.view(np.int16)).pin_memory()
+    idx_h = torch.empty((case.T, k), dtype=torch.int32).pin_memory()
+    gate_h = torch.empty((case.T, k), dtype=torch.float32).pin_memory()
+    counts_h = torch.empty((case.M,), dtype=torch.int32).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(3):
+        mr.more_route_host(Xh, R1h, R2h, k, gate_mode, idx_h, gate_h, counts_h, stream)
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record(stream)
+    for _ in range(e2e_steps):
+        mr.more_route_host(Xh, R1h, R2h, k, gate_mode, idx_h, gate_h, counts_h, stream)
+    ev1.record(stream)
+    stream.synchronize()
+    e2e_secs = ev0.elapsed_time(ev1) * 1e-3
+    if dist:
+        t = torch.tensor([e2e_secs], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_secs = float(t.item())
+    h2d = 2 * (case.T * case.h + case.h * case.r + case.r * case.M)
+    d2h = 8 * case.T * k + 4 * case.M
+    e2e = dict(value=world * case.T * e2e_steps / e2e_secs, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+               steps=e2e_steps, api="more_route_host (pinned host buffers, stream synchronised per call)")
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    roof = roofline(case.T, case.h, case.r, case.M, k, secs / args.steps, peaks, NCU_TRAFFIC_BYTES.get(name))
+    roof["kernel"] = "route_tcgen05_kernel" if mr.more_route_plan(case.T, case.h, case.r, case.M, k).path == 2 else "generic_route_tokens"
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
+                ms_per_step=secs / args.steps * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload=describe(name, case, gate_mode), l2=l2_note,
+                            plan=vars(mr.more_route_plan(case.T, case.h, case.r, case.M, k))),
+                clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roof)
+
+    # ---- context: unfused library-op router on the same inputs
+    ms_unfused = unfused_reference_ms(torch, bufs, case, gate_mode)
+    line["unfused_gpu_reference_ms"] = ms_unfused
+
+    # ---- the CPU oracle on the host cores (a reported baseline, not the target)
+    if world == 1 and not args.no_cpu_baseline:
+        rate, n, dt, cores = oracle_rate(case, gate_mode)
+        line["cpu_baseline"] = dict(value=rate, unit=UNIT, cores=cores, kind="oracle",
+                                    sample=f"first {n} of {case.T} tokens of the workload, {dt:.1f} s, fp64 oracle with OpenMP")
+    else:
+        line["cpu_baseline"] = None
+
+    # ---- per-configuration table (same protocol, fewer steps), context for the headline
+    if world == 1 and not args.no_others:
+        others = {}
+        del bufs
+        torch.cuda.empty_cache()
+        for oname, cfg in inputs.CONFIGS.items():
+            for gm in (0, 1):
+                ocase = inputs.make_config(oname, gate_mode=gm)
+                ocopies, _ = copies_for(ocase)
+                obufs = make_bufs(torch, ocase, ocopies)
+                osecs = time_router(mr, torch, obufs, ocase.k, gm, 200, 50, stream) / 200
+                r = roofline(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k, osecs, peaks)
+                others[f"{oname}/mode{gm}"] = dict(us=osecs * 1e6, tokens_per_s=ocase.T / osecs, bound=r["bound"],
+                                                    roofline_frac=r["frac"],
+                                                    msplit=mr.more_route_plan(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k).msplit)
+                del obufs
+            torch.cuda.empty_cache()
+        line["others"] = others
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

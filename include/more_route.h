@@ -1,0 +1,141 @@
+/*
+ * more_route.h -- C interface of the fused low-rank MoE router for NVIDIA B200 (sm_100a).
+ *
+ * The router scores M experts through an r-dimensional bottleneck and keeps the k best per token
+ * (MoRE layer, Section 2:  g(x) = softmax(TopK(R_1 R_2 x)) ).  Operand names follow this interface, which
+ * stores the paper's factors transposed:
+ *
+ *      X  [T][h]  token activations            (the paper's N = B*T tokens is this T)
+ *      R1 [h][r]  down-projection              (= the paper's R_2 transposed;  z = X R1, Section 3.1 Setup)
+ *      R2 [r][M]  expert vectors as columns    (= the paper's R_1 transposed;  logits l = z R2, Eq. app_logits)
+ *
+ * All three are bfloat16, row-major, contiguous, in DEVICE memory unless an entry point says otherwise.
+ * The logits are produced tile by tile over M and reduced on chip to a per-token running top-k (and, in
+ * full-softmax mode, a running max / sum of exponentials, Eq. app_online), so the T x M logit matrix is never
+ * written to memory (Algorithm 1).  Accumulation is fp32; z is carried into the second contraction as a
+ * bfloat16 high part plus a bfloat16 low part, so the logits are accurate to about 1e-5 rather than to the
+ * 1e-2 a single bfloat16 z would give.
+ *
+ * Every function returns MORE_OK (0) or a negative MORE_ERR_* code.  On an error detected before launch
+ * nothing is launched and no output is touched.  Calls are asynchronous on the given stream unless stated.
+ * Buffers are owned by the caller; the library keeps, per device, one cached scratch allocation (grown on
+ * demand by cudaMalloc, which may synchronise the device the first time a larger problem is seen) and a
+ * small cache of TMA descriptors.  Calls on different host threads are serialised internally; two calls
+ * whose kernels may overlap on the GPU (different streams) must not be issued for the same device, because
+ * they share that scratch.
+ */
+#ifndef MORE_ROUTE_H_
+#define MORE_ROUTE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* gate_mode */
+enum {
+    MORE_GATE_TOPK_SOFTMAX = 0, /* softmax over the k selected logits (Section 2); each row of gates sums to 1 */
+    MORE_GATE_FULL_SOFTMAX = 1  /* P_{n,j} = exp(l_{n,j} - m_n) / Z_n over all M experts (Eq. app_softmax), carried
+                                   across expert tiles by the online recurrence Eq. app_online; the k reported
+                                   entries are NOT renormalised, so a row sums to less than 1 */
+};
+
+/* path selector of more_route_ex */
+enum {
+    MORE_PATH_AUTO = 0,    /* tensor-core path when the shape allows it, otherwise the generic path */
+    MORE_PATH_GENERIC = 1, /* CUDA-core kernels, any shape within the limits below */
+    MORE_PATH_TCGEN05 = 2  /* TMA + tcgen05/TMEM kernel; needs h % 8 == 0, M % 8 == 0, r % 8 == 0, r <= 64, k <= 32 */
+};
+
+/* error codes */
+enum {
+    MORE_OK = 0,
+    MORE_ERR_NULL = -1,    /* a required pointer is NULL */
+    MORE_ERR_SHAPE = -2,   /* T < 0; h, r, M or k < 1; k > M; k > MORE_K_MAX; r > MORE_R_MAX; or the forced path cannot run the shape */
+    MORE_ERR_ALIGN = -3,   /* X, R1 or R2 not 16-byte aligned, or an output not 4-byte aligned */
+    MORE_ERR_MODE = -4,    /* unknown gate_mode or path */
+    MORE_ERR_ARCH = -5,    /* the current device is not compute capability 10.x */
+    MORE_ERR_CUDA = -6,    /* a CUDA runtime/driver call failed (allocation, descriptor encode, launch) */
+    MORE_ERR_TIMEOUT = -7, /* a bounded on-device wait gave up; outputs of that call are undefined (more_route_status) */
+    MORE_ERR_TOO_LARGE = -8 /* problem exceeds a fixed capacity of the chosen entry point */
+};
+
+#define MORE_K_MAX 32     /* largest k */
+#define MORE_R_MAX 1024   /* largest r (generic path); the tensor-core path takes r <= 64 */
+
+/*
+ * more_route -- route T tokens (Algorithm 1 plus the gates of Section 2 / Eq. app_softmax and the per-expert
+ * counts, the bincount of Eq. app_lbal without its 1/(Nk) factor).
+ *
+ *   X, R1, R2   device, bf16, layouts above, 16-byte aligned, read only.  Values must be finite.
+ *   T,h,r,M,k   sizes; 1 <= k <= min(M, MORE_K_MAX).  T == 0 is allowed (only out_counts is written).
+ *   gate_mode   MORE_GATE_*.
+ *   out_idx     device int32 [T][k]: expert ids in [0, M), distinct within a row, ordered by descending logit,
+ *               equal logits by ascending id.
+ *   out_gate    device fp32 [T][k]: gate weights in the same order.
+ *   out_counts  device int32 [M]: OVERWRITTEN with the number of (token, slot) pairs that selected each expert;
+ *               sums to T*k.  (The library zeroes it on `stream` before accumulating.)
+ *   stream      a cudaStream_t (NULL = the legacy default stream).  Outputs are valid once it has been synchronised.
+ */
+int more_route(const void* X, const void* R1, const void* R2,
+               int T, int h, int r, int M, int k, int gate_mode,
+               int32_t* out_idx, float* out_gate, int32_t* out_counts, void* stream);
+
+/*
+ * more_route_ex -- more_route with two optional extra outputs and explicit control of the launch plan.
+ *
+ *   out_topval  device fp32 [T][k] or NULL: the selected logits (Algorithm 1's TopVals), same order as out_idx.
+ *   out_lse     device fp32 [T] or NULL: m_n + log Z_n over all M experts (Eq. app_softmax); computed in either
+ *               gate mode when requested (it forces the full-softmax sweep).
+ *   path        MORE_PATH_*; a forced path that cannot run the shape gives MORE_ERR_SHAPE.
+ *   msplit      tensor-core path only: number of CTAs that share one 128-token block by splitting the expert
+ *               range (partial top-k lists and (m, Z) pairs are merged by the last CTA to finish);
+ *               0 = chosen by the library.  Results do not depend on it.
+ */
+int more_route_ex(const void* X, const void* R1, const void* R2,
+                  int T, int h, int r, int M, int k, int gate_mode,
+                  int32_t* out_idx, float* out_gate, int32_t* out_counts,
+                  float* out_topval, float* out_lse, int path, int msplit, void* stream);
+
+/*
+ * more_route_host -- the same computation for callers whose buffers live in HOST memory (pinned memory makes
+ * the copies asynchronous and faster, pageable memory also works).  The library copies X, R1, R2 to device
+ * staging buffers it owns, runs more_route on `stream`, copies out_idx / out_gate / out_counts back and
+ * SYNCHRONISES the stream before returning, so the outputs are valid on return.
+ * All pointers are host pointers; shapes, modes and errors as for more_route.
+ */
+int more_route_host(const void* X_host, const void* R1_host, const void* R2_host,
+                    int T, int h, int r, int M, int k, int gate_mode,
+                    int32_t* out_idx_host, float* out_gate_host, int32_t* out_counts_host, void* stream);
+
+/*
+ * more_route_plan -- report, without launching, what more_route_ex would do for a shape:
+ *   *path_out   MORE_PATH_GENERIC or MORE_PATH_TCGEN05
+ *   *msplit_out CTAs per 128-token block (1 on the generic path)
+ *   *ctas_out   total CTAs of the main kernel
+ * Any of the three may be NULL.  Host-only; needs no device.
+ */
+int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit,
+                    int* path_out, int* msplit_out, int* ctas_out);
+
+/*
+ * more_route_status -- synchronise `stream` and return the sticky device-side status of the current device:
+ * MORE_OK, or MORE_ERR_TIMEOUT if any kernel since the last call gave up on a bounded wait (an mbarrier that
+ * never completed).  Reading the status clears it.
+ */
+int more_route_status(void* stream);
+
+/* more_route_launches -- number of kernels this library has launched in this process (all devices). */
+long long more_route_launches(void);
+
+/* more_strerror -- a static, human-readable string for a MORE_* code. */
+const char* more_strerror(int code);
+
+/* more_version -- interface version, major*100 + minor. */
+int more_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MORE_ROUTE_H_ */

@@ -1,0 +1,62 @@
+// Internal declarations shared by the translation units of libmore_route.so (not installed).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/more_route.h"
+
+namespace more {
+
+struct RouteArgs {
+    const __nv_bfloat16* X;
+    const __nv_bfloat16* R1;
+    const __nv_bfloat16* R2;
+    int T, h, r, M, k, gate_mode;
+    int32_t* out_idx;
+    float* out_gate;
+    int32_t* out_counts;
+    float* out_topval;  // nullable
+    float* out_lse;     // nullable
+    cudaStream_t stream;
+};
+
+// Per-device state: one cached scratch allocation, the sticky status word, device facts.
+struct DeviceCtx {
+    int dev = -1;
+    int cc_major = 0;
+    int sm_count = 0;
+    void* scratch = nullptr;
+    size_t scratch_bytes = 0;
+    int* status = nullptr;        // device int: 0 = ok, else a MORE_ERR_* code written by a kernel
+    void* staging = nullptr;      // device staging of more_route_host
+    size_t staging_bytes = 0;
+};
+
+// Tokens per CTA of the tensor-core path, and the expert-tile width of one accumulator buffer.
+constexpr int kBlockTokens = 128;
+constexpr int kTileExperts = 128;
+
+// Launch plan (host-only logic, testable without a device).
+struct Plan {
+    int path;     // MORE_PATH_GENERIC or MORE_PATH_TCGEN05
+    int msplit;   // CTAs per token block
+    int ctas;     // CTAs of the main kernel
+    int rpad;     // r rounded up to a multiple of 16 (tensor-core path)
+};
+
+bool tcgen05_shape_ok(int T, int h, int r, int M, int k);
+int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int sm_count, Plan* out);
+
+// Scratch bytes each path needs for a problem.
+size_t generic_scratch_bytes(const RouteArgs& a);
+size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p);
+
+// Launchers: enqueue on a.stream, return MORE_OK / MORE_ERR_*.  `scratch` is at least *_scratch_bytes().
+int launch_generic(const RouteArgs& a, DeviceCtx& ctx, void* scratch);
+int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
+
+void count_launch(int n = 1);
+
+}  // namespace more

@@ -1,0 +1,257 @@
+// Host side of libmore_route.so: argument checks, per-device state, launch planning, the extern "C" entry points.
+#include "more_internal.h"
+
+#include <atomic>
+#include <mutex>
+#include <new>
+
+namespace more {
+
+namespace {
+
+std::mutex g_mutex;
+std::atomic<long long> g_launches{0};
+constexpr int kMaxDevices = 64;
+DeviceCtx g_ctx[kMaxDevices];
+
+int get_ctx(DeviceCtx** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return MORE_ERR_CUDA;
+    DeviceCtx& c = g_ctx[dev];
+    if (c.dev != dev) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return MORE_ERR_CUDA;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MORE_ERR_CUDA;
+        c.cc_major = major;
+        c.sm_count = sms;
+        if (major != 10) return MORE_ERR_ARCH;
+        if (cudaMalloc(&c.status, sizeof(int)) != cudaSuccess) return MORE_ERR_CUDA;
+        if (cudaMemset(c.status, 0, sizeof(int)) != cudaSuccess) return MORE_ERR_CUDA;
+        c.dev = dev;
+    }
+    if (c.cc_major != 10) return MORE_ERR_ARCH;
+    *out = &c;
+    return MORE_OK;
+}
+
+int ensure_bytes(void** buf, size_t* have, size_t need)
+{
+    if (need <= *have) return MORE_OK;
+    if (*buf) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return MORE_ERR_CUDA;   // nothing may still be using it
+        cudaFree(*buf);
+        *buf = nullptr;
+        *have = 0;
+    }
+    size_t bytes = (need + ((size_t)1 << 20) - 1) & ~(((size_t)1 << 20) - 1);
+    if (cudaMalloc(buf, bytes) != cudaSuccess) { cudaGetLastError(); return MORE_ERR_CUDA; }
+    *have = bytes;
+    return MORE_OK;
+}
+
+int check_shape(int T, int h, int r, int M, int k, int gate_mode, int path)
+{
+    if (gate_mode != MORE_GATE_TOPK_SOFTMAX && gate_mode != MORE_GATE_FULL_SOFTMAX) return MORE_ERR_MODE;
+    if (path != MORE_PATH_AUTO && path != MORE_PATH_GENERIC && path != MORE_PATH_TCGEN05) return MORE_ERR_MODE;
+    if (T < 0 || h < 1 || r < 1 || M < 1 || k < 1 || k > M || k > MORE_K_MAX || r > MORE_R_MAX) return MORE_ERR_SHAPE;
+    return MORE_OK;
+}
+
+bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+
+int route_device(const RouteArgs& a, int path, int msplit)
+{
+    int rc = check_shape(a.T, a.h, a.r, a.M, a.k, a.gate_mode, path);
+    if (rc != MORE_OK) return rc;
+    if (!a.out_counts) return MORE_ERR_NULL;
+    if (a.T > 0 && (!a.X || !a.R1 || !a.R2 || !a.out_idx || !a.out_gate)) return MORE_ERR_NULL;
+    if (!aligned(a.X, 16) || !aligned(a.R1, 16) || !aligned(a.R2, 16)) return MORE_ERR_ALIGN;
+    if (!aligned(a.out_idx, 4) || !aligned(a.out_gate, 4) || !aligned(a.out_counts, 4) || !aligned(a.out_topval, 4) ||
+        !aligned(a.out_lse, 4))
+        return MORE_ERR_ALIGN;
+
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    Plan plan;
+    rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, path, msplit, ctx->sm_count, &plan);
+    if (rc != MORE_OK) return rc;
+    const size_t need = plan.path == MORE_PATH_TCGEN05 ? tcgen05_scratch_bytes(a, plan) : generic_scratch_bytes(a);
+    rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, need);
+    if (rc != MORE_OK) return rc;
+    if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) return MORE_ERR_CUDA;
+    if (a.T == 0) return MORE_OK;
+    return plan.path == MORE_PATH_TCGEN05 ? launch_tcgen05(a, *ctx, plan, ctx->scratch)
+                                          : launch_generic(a, *ctx, ctx->scratch);
+}
+
+}  // namespace
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int sm_count, Plan* out)
+{
+    (void)gate_mode;
+    const bool fast_ok = tcgen05_shape_ok(T, h, r, M, k);
+    if (path == MORE_PATH_TCGEN05 && !fast_ok) return MORE_ERR_SHAPE;
+    if (msplit < 0) return MORE_ERR_SHAPE;
+    Plan p;
+    p.rpad = (r + 15) / 16 * 16;
+    if (path == MORE_PATH_GENERIC || !fast_ok) {
+        p.path = MORE_PATH_GENERIC;
+        p.msplit = 1;
+        p.ctas = (T + 7) / 8;
+        *out = p;
+        return MORE_OK;
+    }
+    p.path = MORE_PATH_TCGEN05;
+    const int blocks = (T + kBlockTokens - 1) / kBlockTokens;
+    const int tiles = (M + kTileExperts - 1) / kTileExperts;
+    int s = msplit;
+    if (s == 0) {
+        // Pick the split that minimises (rounds of CTAs over the SMs) x (time of one CTA).  One CTA costs the
+        // z projection (~ h columns of X) plus its share of the expert sweep; weigh a logit column like
+        // `w` X columns (the sweep's per-column cost relative to streaming one X column).
+        if (sm_count <= 0) sm_count = 148;
+        const double w = 1.0;
+        const int slots = 2 * sm_count;                 // two CTAs are resident per SM
+        double best = 1e300;
+        s = 1;
+        for (int c = 1; c <= 64 && c <= tiles; ++c) {
+            const long long ctas = (long long)blocks * c;
+            const double rounds = (double)((ctas + slots - 1) / slots);
+            const double per_cta = 0.25 * h + w * ((tiles + c - 1) / c) * kTileExperts + 512.0;
+            const double cost = rounds * per_cta;
+            if (cost < best * 0.97) { best = cost; s = c; }
+        }
+    }
+    if (s > tiles) s = tiles;
+    if (s < 1) s = 1;
+    if (s > 64) return MORE_ERR_SHAPE;
+    p.msplit = s;
+    p.ctas = blocks * s;
+    *out = p;
+    return MORE_OK;
+}
+
+}  // namespace more
+
+using namespace more;
+
+extern "C" {
+
+int more_route_ex(const void* X, const void* R1, const void* R2, int T, int h, int r, int M, int k, int gate_mode,
+                  int32_t* out_idx, float* out_gate, int32_t* out_counts, float* out_topval, float* out_lse, int path,
+                  int msplit, void* stream)
+{
+    RouteArgs a;
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.R1 = static_cast<const __nv_bfloat16*>(R1);
+    a.R2 = static_cast<const __nv_bfloat16*>(R2);
+    a.T = T; a.h = h; a.r = r; a.M = M; a.k = k; a.gate_mode = gate_mode;
+    a.out_idx = out_idx; a.out_gate = out_gate; a.out_counts = out_counts;
+    a.out_topval = out_topval; a.out_lse = out_lse;
+    a.stream = static_cast<cudaStream_t>(stream);
+    return route_device(a, path, msplit);
+}
+
+int more_route(const void* X, const void* R1, const void* R2, int T, int h, int r, int M, int k, int gate_mode,
+               int32_t* out_idx, float* out_gate, int32_t* out_counts, void* stream)
+{
+    return more_route_ex(X, R1, R2, T, h, r, M, k, gate_mode, out_idx, out_gate, out_counts, nullptr, nullptr,
+                         MORE_PATH_AUTO, 0, stream);
+}
+
+int more_route_host(const void* Xh, const void* R1h, const void* R2h, int T, int h, int r, int M, int k, int gate_mode,
+                    int32_t* idx_h, float* gate_h, int32_t* counts_h, void* stream)
+{
+    int rc = check_shape(T, h, r, M, k, gate_mode, MORE_PATH_AUTO);
+    if (rc != MORE_OK) return rc;
+    if (!counts_h) return MORE_ERR_NULL;
+    if (T > 0 && (!Xh || !R1h || !R2h || !idx_h || !gate_h)) return MORE_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
+    const size_t bX = up((size_t)T * h * 2), bR1 = up((size_t)h * r * 2), bR2 = up((size_t)r * M * 2);
+    const size_t bI = up((size_t)T * k * 4), bG = up((size_t)T * k * 4), bC = up((size_t)M * 4);
+    char* base = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        DeviceCtx* ctx = nullptr;
+        rc = get_ctx(&ctx);
+        if (rc != MORE_OK) return rc;
+        rc = ensure_bytes(&ctx->staging, &ctx->staging_bytes, bX + bR1 + bR2 + bI + bG + bC);
+        if (rc != MORE_OK) return rc;
+        base = static_cast<char*>(ctx->staging);
+    }
+    char* dX = base; char* dR1 = dX + bX; char* dR2 = dR1 + bR1;
+    char* dI = dR2 + bR2; char* dG = dI + bI; char* dC = dG + bG;
+    bool ok = true;
+    if (T > 0) {
+        ok = ok && cudaMemcpyAsync(dX, Xh, (size_t)T * h * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(dR1, R1h, (size_t)h * r * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(dR2, R2h, (size_t)r * M * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
+    }
+    if (!ok) return MORE_ERR_CUDA;
+    rc = more_route(dX, dR1, dR2, T, h, r, M, k, gate_mode, reinterpret_cast<int32_t*>(dI),
+                    reinterpret_cast<float*>(dG), reinterpret_cast<int32_t*>(dC), stream);
+    if (rc != MORE_OK) return rc;
+    if (T > 0) {
+        ok = ok && cudaMemcpyAsync(idx_h, dI, (size_t)T * k * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        ok = ok && cudaMemcpyAsync(gate_h, dG, (size_t)T * k * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    }
+    ok = ok && cudaMemcpyAsync(counts_h, dC, (size_t)M * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(st) == cudaSuccess;
+    return ok ? MORE_OK : MORE_ERR_CUDA;
+}
+
+int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int* path_out,
+                    int* msplit_out, int* ctas_out)
+{
+    int rc = check_shape(T, h, r, M, k, gate_mode, path);
+    if (rc != MORE_OK) return rc;
+    Plan p;
+    rc = make_plan(T, h, r, M, k, gate_mode, path, msplit, 148, &p);
+    if (rc != MORE_OK) return rc;
+    if (path_out) *path_out = p.path;
+    if (msplit_out) *msplit_out = p.msplit;
+    if (ctas_out) *ctas_out = p.ctas;
+    return MORE_OK;
+}
+
+int more_route_status(void* stream)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int host = 0;
+    if (cudaMemcpyAsync(&host, ctx->status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MORE_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->status, 0, sizeof(int), st) != cudaSuccess) return MORE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MORE_ERR_CUDA;
+    return host == 0 ? MORE_OK : MORE_ERR_TIMEOUT;
+}
+
+long long more_route_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+const char* more_strerror(int code)
+{
+    switch (code) {
+        case MORE_OK: return "ok";
+        case MORE_ERR_NULL: return "a required pointer is NULL";
+        case MORE_ERR_SHAPE: return "unsupported shape (sizes out of range, k > M, or the forced path cannot run it)";
+        case MORE_ERR_ALIGN: return "misaligned pointer (inputs need 16 bytes, outputs 4)";
+        case MORE_ERR_MODE: return "unknown gate_mode or path";
+        case MORE_ERR_ARCH: return "the current device is not compute capability 10.x (B200)";
+        case MORE_ERR_CUDA: return "a CUDA call failed";
+        case MORE_ERR_TIMEOUT: return "a bounded on-device wait gave up";
+        case MORE_ERR_TOO_LARGE: return "problem exceeds the fixed capacity of this entry point";
+        default: return "unknown error code";
+    }
+}
+
+int more_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,684 @@
+// Tensor-core path of the fused low-rank router for sm_100a: TMA-staged operands, tcgen05.mma with TMEM
+// accumulators, a thread-per-token epilogue that keeps the running top-k (and, on request, the online
+// (max, sum-of-exponentials) pair of Eq. app_online) in registers.
+//
+// One CTA routes one block of 128 tokens over one contiguous range of expert tiles (Algorithm 1, with the token
+// block additionally split over `msplit` CTAs along the expert dimension):
+//
+//   phase 1  z = X_blk R1            TMA streams 128x64 X tiles and 64x64 R1 tiles (zero-filled beyond r),
+//                                    tcgen05.mma accumulates the 128 x 64 fp32 block in TMEM.
+//   narrow   z -> bf16 hi + bf16 lo  written to shared memory as the K-major A operand [hi | lo].  Carrying both
+//                                    parts keeps the logits within ~3e-5 of exact arithmetic.
+//   phase 2  y = z R2[:, tile]       one 128-expert tile at a time: TMA brings the r x 128 slice of R2, tcgen05.mma
+//                                    (hi then lo into the same accumulator) fills one of two TMEM buffers while
+//                                    the epilogue drains the other: TMEM lane = token, so each epilogue thread owns
+//                                    one token and reads its logits 32 columns at a time.
+//   merge    running top-k           sorted (value, id) list in registers; a chunk is looked at element by element
+//                                    only if its maximum beats the list's last entry.
+//   finish   gates, ids, counts      written by the CTA itself (msplit == 1) or, after the partial lists have been
+//                                    parked in scratch, by whichever CTA of the token block finishes last.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue (warp w reads
+// TMEM lanes 32*(w%4)..).  Two CTAs are resident per SM (256 TMEM columns and ~100 KB of shared memory each), so
+// one CTA's HBM-bound phase 1 overlaps the other's expert sweep.
+//
+// Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
+// status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
+#include "more_internal.h"
+
+#include <cuda.h>   // CUtensorMap and the driver entry-point typedef only; libcuda is resolved at run time
+#include <limits.h>
+
+namespace more {
+
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kEpilogueThreads = 128;
+constexpr int kStagesP1 = 4;                       // phase-1 ring: 16 KB of X + 8 KB of R1 per stage
+constexpr int kXTileBytes = kBlockTokens * 128;    // 128 tokens x 64 bf16
+constexpr int kR1TileBytes = 64 * 128;             // 64 K-rows x 64 bf16 (columns >= r are zero-filled by TMA)
+constexpr int kP1StageBytes = kXTileBytes + kR1TileBytes;
+constexpr int kRingBytes = kStagesP1 * kP1StageBytes;   // 96 KB, reused by phase 2
+constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
+constexpr int kTmemCols = 256;                     // two 128-column fp32 accumulator buffers
+constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s
+
+// ------------------------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of budget).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > kWaitBudgetCycles) {
+                *abort_flag = 1;
+                atomicExch(status, MORE_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// 32 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15]), "=r"(u[16]),
+          "=r"(u[17]), "=r"(u[18]), "=r"(u[19]), "=r"(u[20]), "=r"(u[21]), "=r"(u[22]), "=r"(u[23]), "=r"(u[24]),
+          "=r"(u[25]), "=r"(u[26]), "=r"(u[27]), "=r"(u[28]), "=r"(u[29]), "=r"(u[30]), "=r"(u[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
+{
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3]), "=r"(u[4]), "=r"(u[5]), "=r"(u[6]), "=r"(u[7]), "=r"(u[8]),
+          "=r"(u[9]), "=r"(u[10]), "=r"(u[11]), "=r"(u[12]), "=r"(u[13]), "=r"(u[14]), "=r"(u[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ float ex2f(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// ------------------------------------------------------------------------------------------- UMMA descriptors
+// Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
+//   K-major operand  (rows = M/N index, 128-byte rows of 64 bf16 along K): SBO = 1024 B between 8-row groups.
+//   MN-major operand (rows = K index, 128-byte rows of 64 bf16 along M/N): SBO = 1024 B between 8-K-row groups,
+//                     LBO = distance between successive 64-element column blocks.
+__device__ __forceinline__ uint64_t umma_desc_sw128(uint32_t smem_addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;     // descriptor version
+    d |= (uint64_t)2 << 61;     // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: D = fp32, A = B = bf16, A K-major, B MN-major, M = 128, given N.
+__host__ __device__ constexpr uint32_t umma_idesc(int n)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
+
+// -------------------------------------------------------------------------------------------- running top-k
+template <int KCAP>
+struct TopList {
+    float v[KCAP];
+    int id[KCAP];
+    __device__ __forceinline__ void init()
+    {
+#pragma unroll
+        for (int s = 0; s < KCAP; ++s) { v[s] = -INFINITY; id[s] = INT_MAX; }
+    }
+    __device__ __forceinline__ float tau() const { return v[KCAP - 1]; }
+    // Insert (x, j) with x > tau().  Equal values keep the earlier (smaller-id) entry ahead.
+    __device__ __forceinline__ void insert(float x, int j)
+    {
+#pragma unroll
+        for (int s = KCAP - 1; s > 0; --s) {
+            const bool above_prev = x > v[s - 1];
+            const bool above_this = x > v[s];
+            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
+            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
+        }
+        const bool top = x > v[0];
+        v[0] = top ? x : v[0];
+        id[0] = top ? j : id[0];
+    }
+};
+
+struct KernelParams {
+    int T, h, r, M, k, gate_mode, msplit;
+    int tiles_total;             // ceil(M / 128)
+    int32_t* out_idx;
+    float* out_gate;
+    int32_t* out_counts;
+    float* out_topval;
+    float* out_lse;
+    int* status;
+    // scratch (msplit > 1): per token block an arrival counter, per (token, split) a partial list and (m, Z)
+    unsigned* counters;
+    float* part_val;
+    int* part_id;
+    float2* part_mz;
+};
+
+// Final outputs of one token from its sorted list and (m2, z): m2 is the running max in log2 units.
+template <int KCAP>
+__device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, const TopList<KCAP>& L, float m2,
+                                            float zsum)
+{
+    constexpr float kLn2 = 0.6931471805599453f, kLog2e = 1.4426950408889634f;
+    const int k = p.k;
+    float denom = 0.f;
+    if (p.gate_mode == MORE_GATE_TOPK_SOFTMAX) {
+#pragma unroll
+        for (int q = 0; q < KCAP; ++q)
+            if (q < k) denom += ex2f((L.v[q] - L.v[0]) * kLog2e);
+    } else {
+        denom = zsum;
+    }
+    const float inv = 1.f / denom;
+    const float ref2 = (p.gate_mode == MORE_GATE_TOPK_SOFTMAX) ? L.v[0] * kLog2e : m2;
+#pragma unroll
+    for (int q = 0; q < KCAP; ++q) {
+        if (q < k) {
+            p.out_idx[row * k + q] = L.id[q];
+            p.out_gate[row * k + q] = ex2f(L.v[q] * kLog2e - ref2) * inv;
+            if (p.out_topval) p.out_topval[row * k + q] = L.v[q];
+            atomicAdd(p.out_counts + L.id[q], 1);
+        }
+    }
+    if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
+}
+
+// ------------------------------------------------------------------------------------------------- the kernel
+template <int RPAD, int KCAP, bool LSE>
+__global__ void __launch_bounds__(kThreads, 2)
+route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
+                     const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
+{
+    constexpr int kKSteps = RPAD / 16;                       // UMMA K = 16
+    constexpr int kZopBytes = (RPAD == 64) ? 32768 : 16384;  // [hi | lo] rows of 128 B; two slabs when 2*RPAD > 64
+    constexpr int kR2StageBytes = RPAD * 256;                // two 64-expert blocks of RPAD rows x 128 B
+    constexpr int kStagesP2 = ((kRingBytes - kZopBytes) / kR2StageBytes) > 8 ? 8 : ((kRingBytes - kZopBytes) / kR2StageBytes);
+    constexpr float kLog2e = 1.4426950408889634f;
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = (raw + 1023u) & ~1023u;            // 1024-aligned: the 128-B swizzle repeats every 1 KB
+    uint8_t* ring_ptr = smem_raw + (ring - raw);
+    uint8_t* ctl = ring_ptr + kRingBytes;                    // control block
+    uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
+    // barrier slots
+    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kStagesP1, B_ZACC = B_EMPTY1 + kStagesP1, B_ZOP = B_ZACC + 1,
+                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
+                  B_COUNT = B_ACCE + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
+    int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
+    const uint32_t bar0 = smem_u32(bars);
+    auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int blk = blockIdx.x / p.msplit, split = blockIdx.x % p.msplit;
+    const int tok0 = blk * kBlockTokens;
+    // expert tiles of this CTA: an even share of ceil(M/128) tiles
+    const int tile_lo = (int)(((long long)p.tiles_total * split) / p.msplit);
+    const int tile_hi = (int)(((long long)p.tiles_total * (split + 1)) / p.msplit);
+    const int ntiles = tile_hi - tile_lo;
+    const int ktiles1 = (p.h + 63) / 64;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < kStagesP1; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
+        mbar_init(bar(B_ZACC), 1);
+        mbar_init(bar(B_ZOP), kEpilogueThreads);
+        for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads); }
+        *abort_flag = 0;
+        *last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const uint32_t zop = ring;                        // phase 2: A operand [hi | lo]
+    const uint32_t r2ring = ring + kZopBytes;         // phase 2: R2 stages
+
+    if (warp == 0) {
+        // ===================================================================================== TMA producer
+        if (lane == 0) {
+            bool ok = true;
+            for (int kt = 0; kt < ktiles1 && ok; ++kt) {
+                const int s = kt % kStagesP1;
+                if (kt >= kStagesP1) ok = mbar_wait(bar(B_EMPTY1 + s), ((kt / kStagesP1) - 1) & 1, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t dst = ring + s * kP1StageBytes;
+                mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
+                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);
+                tma_load_2d(dst + kXTileBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
+            }
+            // the ring is reused by phase 2: wait until every phase-1 MMA has finished reading it
+            ok = ok && mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
+            for (int it = 0; it < ntiles && ok; ++it) {
+                const int s = it % kStagesP2;
+                if (it >= kStagesP2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it / kStagesP2) - 1) & 1, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t dst = r2ring + s * kR2StageBytes;
+                const int e0 = (tile_lo + it) * kTileExperts;
+                mbar_expect_tx(bar(B_FULL2 + s), kR2StageBytes);
+                tma_load_2d(dst, &map_r2, bar(B_FULL2 + s), e0, 0);
+                tma_load_2d(dst + RPAD * 128, &map_r2, bar(B_FULL2 + s), e0 + 64, 0);
+            }
+        }
+    } else if (warp == 1) {
+        // ======================================================================================= MMA issuer
+        if (lane == 0) {
+            bool ok = true;
+            constexpr uint32_t idesc1 = umma_idesc(64);
+            constexpr uint32_t idesc2 = umma_idesc(kTileExperts);
+            for (int kt = 0; kt < ktiles1 && ok; ++kt) {
+                const int s = kt % kStagesP1;
+                ok = mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t xa = ring + s * kP1StageBytes, rb = xa + kXTileBytes;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {
+                    const uint64_t ad = umma_desc_sw128(xa + kk * 32, 16, 1024);            // K-major, +32 B per K=16
+                    const uint64_t bd = umma_desc_sw128(rb + kk * 2048, 8192, 1024);        // MN-major, 16 K-rows
+                    tc_mma_bf16(tmem_base, ad, bd, idesc1, (kt | kk) != 0);
+                }
+                tc_commit(bar(B_EMPTY1 + s));
+            }
+            if (ok) tc_commit(bar(B_ZACC));
+            ok = ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status);
+            tc_fence_after();
+            for (int it = 0; it < ntiles && ok; ++it) {
+                const int s = it % kStagesP2, b = it & 1;
+                ok = mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status);
+                ok = ok && mbar_wait(bar(B_ACCE + b), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t rb = r2ring + s * kR2StageBytes;
+#pragma unroll
+                for (int j = 0; j < 2 * kKSteps; ++j) {
+                    const uint32_t abyte = j * 32;                                           // K offset in [hi | lo]
+                    const uint64_t ad = umma_desc_sw128(zop + (abyte >> 7) * 16384 + (abyte & 127), 16, 1024);
+                    const uint64_t bd = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
+                    tc_mma_bf16(tmem_base + b * kTileExperts, ad, bd, idesc2, j != 0);
+                }
+                tc_commit(bar(B_EMPTY2 + s));
+                tc_commit(bar(B_ACCF + b));
+            }
+        }
+    } else {
+        // ========================================================================================= epilogue
+        const int q = warp & 3;                              // TMEM lane group this warp may read
+        const int row_in_blk = q * 32 + lane;
+        const int64_t row = (int64_t)tok0 + row_in_blk;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+        bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
+        if (ok) {
+            // ---- narrow z to [hi | lo] and store it as the K-major, 128-B-swizzled A operand
+            tc_fence_after();
+            uint8_t* zrow = ring_ptr + row_in_blk * 128;
+#pragma unroll
+            for (int c = 0; c < RPAD / 16; ++c) {
+                float z[16];
+                tmem_ld16(t_lane + c * 16, z);
+                tmem_ld_wait();
+                uint32_t hi[8], lo[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
+                    const __nv_bfloat16 l0 = __float2bfloat16_rn(z[2 * e] - __bfloat162float(h0));
+                    const __nv_bfloat16 l1 = __float2bfloat16_rn(z[2 * e + 1] - __bfloat162float(h1));
+                    hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                    lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                }
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    // 16-byte chunk `ch` of the logical row [hi(RPAD) | lo(RPAD)]
+                    const int ch_hi = c * 2 + half, ch_lo = RPAD / 8 + c * 2 + half;
+                    const int slab_hi = ch_hi >> 3, slab_lo = ch_lo >> 3;
+                    uint4 vh = make_uint4(hi[half * 4], hi[half * 4 + 1], hi[half * 4 + 2], hi[half * 4 + 3]);
+                    uint4 vl = make_uint4(lo[half * 4], lo[half * 4 + 1], lo[half * 4 + 2], lo[half * 4 + 3]);
+                    *reinterpret_cast<uint4*>(zrow + slab_hi * 16384 + (((ch_hi & 7) ^ (row_in_blk & 7)) << 4)) = vh;
+                    *reinterpret_cast<uint4*>(zrow + slab_lo * 16384 + (((ch_lo & 7) ^ (row_in_blk & 7)) << 4)) = vl;
+                }
+            }
+            fence_async_smem();
+            tc_fence_before();
+            mbar_arrive(bar(B_ZOP));
+        }
+
+        TopList<KCAP> L;
+        L.init();
+        float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
+        for (int it = 0; it < ntiles && ok; ++it) {
+            const int b = it & 1;
+            ok = mbar_wait(bar(B_ACCF + b), (it >> 1) & 1, abort_flag, p.status);
+            if (!ok) break;
+            tc_fence_after();
+            const int e0 = (tile_lo + it) * kTileExperts;
+            const bool ragged = e0 + kTileExperts > p.M;
+#pragma unroll 1
+            for (int c = 0; c < kTileExperts / 32; ++c) {
+                float v[32];
+                tmem_ld32(t_lane + b * kTileExperts + c * 32, v);
+                tmem_ld_wait();
+                const int col0 = e0 + c * 32;
+                if (ragged) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (col0 + i >= p.M) v[i] = -INFINITY;
+                }
+                // chunk maximum: 3-input max tree
+                float t[11];
+#pragma unroll
+                for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+                t[10] = fmaxf(v[30], v[31]);
+                const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
+                const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
+                if (LSE) {
+                    const float c2 = cmax * kLog2e;
+                    if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        a0 += ex2f(fmaf(v[i], kLog2e, -m2));
+                        a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
+                        a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
+                        a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+                    }
+                    zsum += (a0 + a1) + (a2 + a3);
+                }
+                if (cmax > L.tau()) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (v[i] > L.tau()) L.insert(v[i], col0 + i);
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(B_ACCE + b));
+        }
+
+        // ---- finish.  All 128 epilogue threads meet here, also after an abort, so the decision is uniform.
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (*abort_flag == 0) {
+            if (p.msplit == 1) {
+                if (row < p.T) write_token<KCAP>(p, row, L, m2, zsum);
+            } else {
+                // park the partial list; the CTA that arrives last for this token block merges all of them
+                const int64_t slot = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit + split;
+#pragma unroll
+                for (int s = 0; s < KCAP; ++s) {
+                    p.part_val[slot * KCAP + s] = L.v[s];
+                    p.part_id[slot * KCAP + s] = L.id[s];
+                }
+                p.part_mz[slot] = make_float2(m2, zsum);
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (threadIdx.x == 64) {
+                    const unsigned prev = atomicAdd(p.counters + blk, 1u);
+                    *last_flag = (prev == (unsigned)p.msplit - 1u);
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (*last_flag) {
+                    __threadfence();
+                    const int64_t base = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit;
+                    TopList<KCAP> G;
+                    G.init();
+                    float gm = -INFINITY, gz = 0.f;
+                    for (int sp = 0; sp < p.msplit; ++sp) {       // ascending expert ranges: ties keep the smaller id
+                        for (int s = 0; s < KCAP; ++s) {
+                            const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
+                            const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
+                            if (x > G.tau()) G.insert(x, j); else break;   // each partial list is sorted
+                        }
+                        const float2 mz = __ldcg(p.part_mz + base + sp);
+                        if (LSE && mz.x > -INFINITY) {
+                            const float nm = fmaxf(gm, mz.x);
+                            gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
+                            gm = nm;
+                        }
+                    }
+                    if (row < p.T) write_token<KCAP>(p, row, G, gm, gz);
+                    if (threadIdx.x == 64) p.counters[blk] = 0;   // ready for the next call
+                }
+            }
+        }
+    }
+
+    // ---- common exit: everyone arrives here, also after an abort
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag && threadIdx.x == 0) {
+        // give bulk copies that may still be in flight time to land before shared memory is released
+        for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// 2-D bf16 row-major tensor [rows][cols], box = box_cols x box_rows, 128-byte swizzle, zero fill out of bounds.
+struct MapKey {
+    const void* ptr;
+    int rows, cols, box_rows, box_cols;
+    bool operator==(const MapKey& o) const
+    {
+        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows && box_cols == o.box_cols;
+    }
+};
+constexpr int kMapCache = 128;
+MapKey g_keys[kMapCache];
+CUtensorMap g_maps[kMapCache];
+int g_map_count = 0, g_map_next = 0;
+
+int get_map(const void* ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMap* out)
+{
+    const MapKey key{ptr, rows, cols, box_rows, box_cols};
+    for (int i = 0; i < g_map_count; ++i)
+        if (g_keys[i] == key) { *out = g_maps[i]; return MORE_OK; }
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return MORE_ERR_CUDA;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUtensorMap m;
+    CUresult res = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (res != CUDA_SUCCESS) return MORE_ERR_CUDA;
+    const int slot = (g_map_count < kMapCache) ? g_map_count++ : (g_map_next++ % kMapCache);
+    g_keys[slot] = key;
+    g_maps[slot] = m;
+    *out = m;
+    return MORE_OK;
+}
+
+template <int RPAD, int KCAP, bool LSE>
+int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp, int ctas,
+               cudaStream_t st)
+{
+    static unsigned long long configured = 0;   // one bit per device, per instantiation; guarded by the API mutex
+    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE>;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!(configured >> (dev & 63) & 1ull)) {
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+            return MORE_ERR_CUDA;
+        configured |= 1ull << (dev & 63);
+    }
+    kern<<<ctas, kThreads, kSmemBytes, st>>>(mx, m1, m2, kp);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
+
+template <int RPAD, int KCAP>
+int launch_lse(bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp,
+               int ctas, cudaStream_t st)
+{
+    return lse ? launch_one<RPAD, KCAP, true>(mx, m1, m2, kp, ctas, st)
+               : launch_one<RPAD, KCAP, false>(mx, m1, m2, kp, ctas, st);
+}
+
+template <int RPAD>
+int launch_kcap(int k, bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2,
+                const KernelParams& kp, int ctas, cudaStream_t st)
+{
+    if (k <= 8) return launch_lse<RPAD, 8>(lse, mx, m1, m2, kp, ctas, st);
+    if (k <= 16) return launch_lse<RPAD, 16>(lse, mx, m1, m2, kp, ctas, st);
+    return launch_lse<RPAD, 32>(lse, mx, m1, m2, kp, ctas, st);
+}
+
+int kcap_of(int k) { return k <= 8 ? 8 : (k <= 16 ? 16 : 32); }
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+bool tcgen05_shape_ok(int T, int h, int r, int M, int k)
+{
+    return T >= 1 && h % 8 == 0 && M % 8 == 0 && r % 8 == 0 && r <= 64 && k <= 32;
+}
+
+size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p)
+{
+    if (p.msplit <= 1) return 0;
+    const size_t blocks = (size_t)(a.T + kBlockTokens - 1) / kBlockTokens;
+    const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
+    const size_t kc = (size_t)kcap_of(a.k);
+    return align_up(blocks * 4, 256) + align_up(slots * kc * 4, 256) * 2 + align_up(slots * 8, 256);
+}
+
+int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
+{
+    CUtensorMap mx, m1, m2;
+    int rc = get_map(a.X, a.T, a.h, kBlockTokens, 64, &mx);
+    if (rc == MORE_OK) rc = get_map(a.R1, a.h, a.r, 64, 64, &m1);
+    const int rpad = (a.r <= 16) ? 16 : (a.r <= 32 ? 32 : 64);
+    if (rc == MORE_OK) rc = get_map(a.R2, a.r, a.M, rpad, 64, &m2);
+    if (rc != MORE_OK) return rc;
+
+    KernelParams kp;
+    kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
+    kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
+    kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
+    kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
+    kp.status = ctx.status;
+    kp.counters = nullptr; kp.part_val = nullptr; kp.part_id = nullptr; kp.part_mz = nullptr;
+    if (p.msplit > 1) {
+        const size_t blocks = (size_t)(a.T + kBlockTokens - 1) / kBlockTokens;
+        const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
+        const size_t kc = (size_t)kcap_of(a.k);
+        char* base = static_cast<char*>(scratch);
+        kp.counters = reinterpret_cast<unsigned*>(base);
+        base += align_up(blocks * 4, 256);
+        kp.part_val = reinterpret_cast<float*>(base);
+        base += align_up(slots * kc * 4, 256);
+        kp.part_id = reinterpret_cast<int*>(base);
+        base += align_up(slots * kc * 4, 256);
+        kp.part_mz = reinterpret_cast<float2*>(base);
+        if (cudaMemsetAsync(kp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
+    }
+    const bool lse = (a.gate_mode == MORE_GATE_FULL_SOFTMAX) || (a.out_lse != nullptr);
+    switch (rpad) {
+        case 16: return launch_kcap<16>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
+        case 32: return launch_kcap<32>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
+        default: return launch_kcap<64>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
+    }
+}
+
+}  // namespace more
