@@ -146,6 +146,29 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// Wait for outstanding TMEM loads and tie the 32 destination registers to the wait, so that no use of them can be
+// scheduled ahead of it.
+__device__ __forceinline__ void tmem_ld_wait32(float (&v)[32])
+{
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
+                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15]),
+                   "+r"(u[16]), "+r"(u[17]), "+r"(u[18]), "+r"(u[19]), "+r"(u[20]), "+r"(u[21]), "+r"(u[22]),
+                   "+r"(u[23]), "+r"(u[24]), "+r"(u[25]), "+r"(u[26]), "+r"(u[27]), "+r"(u[28]), "+r"(u[29]),
+                   "+r"(u[30]), "+r"(u[31])
+                 :
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait16(float (&v)[16])
+{
+    uint32_t* u = reinterpret_cast<uint32_t*>(v);
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]), "+r"(u[4]), "+r"(u[5]), "+r"(u[6]), "+r"(u[7]),
+                   "+r"(u[8]), "+r"(u[9]), "+r"(u[10]), "+r"(u[11]), "+r"(u[12]), "+r"(u[13]), "+r"(u[14]), "+r"(u[15])
+                 :
+                 : "memory");
+}
 
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
@@ -209,6 +232,83 @@ struct TopList {
     }
 };
 
+// Running top-k of one token.  Between refreshes the sorted list is left alone: elements that beat the cached
+// threshold `tau` (the list's last entry as of the last refresh) are only appended, in ascending column order, to
+// this thread's column of a shared-memory candidate buffer (one predicated 8-byte store each); refresh() then
+// inserts them one by one.  Control flow around the appends is warp-uniform (votes), so the 32 tokens of a warp
+// never serialise on one another's hits, and the inserts of several chunks are executed together.
+constexpr int kCandCap = 16;                              // candidate slots per token
+constexpr int kCandSlotStride = kBlockTokens * 8;         // bytes between successive slots of one token
+constexpr int kCandBytes = kCandCap * kCandSlotStride;
+constexpr int kRefreshAt = 2;                             // refresh a warp after a tile once some token holds this many
+constexpr unsigned kFullMask = 0xffffffffu;
+
+template <int KCAP>
+struct Selector {
+    TopList<KCAP> L;
+    float tau;
+    uint32_t ptr;     // shared-memory address of this thread's next free candidate slot
+    uint32_t base;    // its first slot
+    uint32_t lim;     // ptr is clamped here after every triple; reaching it means "may have lost candidates"
+
+    __device__ __forceinline__ void init(uint32_t first_slot)
+    {
+        L.init();
+        tau = -INFINITY;
+        base = ptr = first_slot;
+        lim = first_slot + (kCandCap - 3) * kCandSlotStride;
+    }
+    __device__ __forceinline__ void refresh()
+    {
+        for (uint32_t a = base; a < ptr; a += kCandSlotStride) {
+            float x;
+            int j;
+            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=f"(x), "=r"(j) : "r"(a) : "memory");
+            L.insert(x, j);
+        }
+        ptr = base;
+        tau = L.tau();
+    }
+    // if (x > tau) append (x, col)
+    __device__ __forceinline__ void append_if_above(float x, int col)
+    {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.gt.f32 p, %1, %3;\n\t"
+            "@p st.shared.v2.b32 [%0], {%1, %2};\n\t"
+            "@p add.u32 %0, %0, %4;\n\t}"
+            : "+r"(ptr)
+            : "f"(x), "r"(col), "f"(tau), "n"(kCandSlotStride)
+            : "memory");
+    }
+    // v: 32 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]); t[10] covers v[30], v[31].
+    // Called by all 32 lanes.  Every element above tau is appended, or, if some token's buffer could not take
+    // them all, the whole warp folds its buffers into the lists and inserts this chunk's elements directly.
+    __device__ __forceinline__ void scan(const float (&v)[32], const float (&t)[11], int col0)
+    {
+        const uint32_t mark = ptr;
+#pragma unroll
+        for (int i = 0; i < 11; ++i) {
+            if (__any_sync(kFullMask, t[i] > tau)) {
+#pragma unroll
+                for (int e = 0; e < 3; ++e) {
+                    const int pos = 3 * i + e;
+                    if (pos < 32) append_if_above(v[pos], col0 + pos);
+                }
+                ptr = min(ptr, lim);
+            }
+        }
+        if (__any_sync(kFullMask, ptr >= lim)) {
+            ptr = mark;                      // forget this chunk's appends (all tokens of the warp) ...
+            refresh();                       // ... fold the older candidates into the lists ...
+#pragma unroll
+            for (int i = 0; i < 32; ++i)     // ... and take this chunk element by element
+                if (v[i] > L.tau()) L.insert(v[i], col0 + i);
+            tau = L.tau();
+        }
+    }
+};
+
 struct KernelParams {
     int T, h, r, M, k, gate_mode, msplit;
     int tiles_total;             // ceil(M / 128)
@@ -263,7 +363,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kKSteps = RPAD / 16;                       // UMMA K = 16
     constexpr int kZopBytes = (RPAD == 64) ? 32768 : 16384;  // [hi | lo] rows of 128 B; two slabs when 2*RPAD > 64
     constexpr int kR2StageBytes = RPAD * 256;                // two 64-expert blocks of RPAD rows x 128 B
-    constexpr int kStagesP2 = ((kRingBytes - kZopBytes) / kR2StageBytes) > 8 ? 8 : ((kRingBytes - kZopBytes) / kR2StageBytes);
+    constexpr int kP2Free = kRingBytes - kZopBytes - kCandBytes;
+    constexpr int kStagesP2 = (kP2Free / kR2StageBytes) > 8 ? 8 : (kP2Free / kR2StageBytes);
+    static_assert(kStagesP2 >= 2, "R2 ring needs at least two stages");
     constexpr float kLog2e = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
@@ -312,7 +414,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t zop = ring;                        // phase 2: A operand [hi | lo]
-    const uint32_t r2ring = ring + kZopBytes;         // phase 2: R2 stages
+    const uint32_t r2ring = ring + kZopBytes + kCandBytes;   // phase 2: R2 stages (after the candidate buffers)
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
@@ -396,7 +498,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
                 tmem_ld16(t_lane + c * 16, z);
-                tmem_ld_wait();
+                tmem_ld_wait16(z);
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
@@ -422,56 +524,80 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             mbar_arrive(bar(B_ZOP));
         }
 
-        TopList<KCAP> L;
-        L.init();
+        Selector<KCAP> S;
+        S.init(ring + kZopBytes + row_in_blk * 8);
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
+
+        // One 32-column chunk: triple maxima, optional online softmax update, candidate scan.
+        auto process = [&](float (&v)[32], int col0, bool ragged) {
+            if (ragged) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i)
+                    if (col0 + i >= p.M) v[i] = -INFINITY;
+            }
+            float t[11];
+#pragma unroll
+            for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+            t[10] = fmaxf(v[30], v[31]);
+            const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
+            const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
+            if (LSE) {
+                const float c2 = cmax * kLog2e;
+                if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; i += 4) {
+                    a0 += ex2f(fmaf(v[i], kLog2e, -m2));
+                    a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
+                    a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
+                    a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+                }
+                zsum += (a0 + a1) + (a2 + a3);
+            }
+            if (__any_sync(kFullMask, cmax > S.tau)) S.scan(v, t, col0);
+        };
+
+        // `ok` is kept warp-uniform from here on (the votes above need all 32 lanes).
+        ok = __all_sync(kFullMask, ok);
+        float va[32], vb[32];
+        if (ok && ntiles > 0) {
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + 0), 0, abort_flag, p.status));
+            if (ok) {
+                tc_fence_after();
+                tmem_ld32(t_lane, va);
+            }
+        }
         for (int it = 0; it < ntiles && ok; ++it) {
             const int b = it & 1;
-            ok = mbar_wait(bar(B_ACCF + b), (it >> 1) & 1, abort_flag, p.status);
-            if (!ok) break;
-            tc_fence_after();
+            const uint32_t tb = t_lane + b * kTileExperts;
             const int e0 = (tile_lo + it) * kTileExperts;
             const bool ragged = e0 + kTileExperts > p.M;
 #pragma unroll 1
-            for (int c = 0; c < kTileExperts / 32; ++c) {
-                float v[32];
-                tmem_ld32(t_lane + b * kTileExperts + c * 32, v);
-                tmem_ld_wait();
-                const int col0 = e0 + c * 32;
-                if (ragged) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (col0 + i >= p.M) v[i] = -INFINITY;
-                }
-                // chunk maximum: 3-input max tree
-                float t[11];
-#pragma unroll
-                for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                t[10] = fmaxf(v[30], v[31]);
-                const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
-                const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
-                if (LSE) {
-                    const float c2 = cmax * kLog2e;
-                    if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
-                        a0 += ex2f(fmaf(v[i], kLog2e, -m2));
-                        a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
-                        a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
-                        a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+            for (int half = 0; half < 2; ++half) {
+                tmem_ld_wait32(va);
+                tmem_ld32(tb + half * 64 + 32, vb);
+                process(va, e0 + half * 64, ragged);
+                tmem_ld_wait32(vb);
+                if (half == 0) {
+                    tmem_ld32(tb + 64, va);
+                } else {
+                    tc_fence_before();
+                    mbar_arrive(bar(B_ACCE + b));            // this accumulator buffer may be overwritten now
+                    if (it + 1 < ntiles) {                   // start on the next tile before finishing this one
+                        ok = __all_sync(kFullMask,
+                                        mbar_wait(bar(B_ACCF + (b ^ 1)), ((it + 1) >> 1) & 1, abort_flag, p.status));
+                        if (ok) {
+                            tc_fence_after();
+                            tmem_ld32(t_lane + (b ^ 1) * kTileExperts, va);
+                        }
                     }
-                    zsum += (a0 + a1) + (a2 + a3);
                 }
-                if (cmax > L.tau()) {
-#pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (v[i] > L.tau()) L.insert(v[i], col0 + i);
-                }
+                process(vb, e0 + half * 64 + 32, ragged);
             }
-            tc_fence_before();
-            mbar_arrive(bar(B_ACCE + b));
+            if (__any_sync(kFullMask, S.ptr >= S.base + kRefreshAt * kCandSlotStride)) S.refresh();
         }
+        S.refresh();
+        TopList<KCAP>& L = S.L;
 
         // ---- finish.  All 128 epilogue threads meet here, also after an abort, so the decision is uniform.
         asm volatile("bar.sync 1, 128;" ::: "memory");
