@@ -89,7 +89,7 @@ int more_route(const void* X, const void* R1, const void* R2,
  *   out_lse     device fp32 [T] or NULL: m_n + log Z_n over all M experts (Eq. app_softmax); computed in either
  *               gate mode when requested (it forces the full-softmax sweep).
  *   path        MORE_PATH_*; a forced path that cannot run the shape gives MORE_ERR_SHAPE.
- *   msplit      tensor-core path only: number of CTAs that share one 128-token block by splitting the expert
+ *   msplit      tensor-core path only: number of CTAs that share one 256-token block by splitting the expert
  *               range (partial top-k lists and (m, Z) pairs are merged by the last CTA to finish);
  *               0 = chosen by the library.  Results do not depend on it.
  */
@@ -112,7 +112,7 @@ int more_route_host(const void* X_host, const void* R1_host, const void* R2_host
 /*
  * more_route_plan -- report, without launching, what more_route_ex would do for a shape:
  *   *path_out   MORE_PATH_GENERIC or MORE_PATH_TCGEN05
- *   *msplit_out CTAs per 128-token block (1 on the generic path)
+ *   *msplit_out CTAs per 256-token block (1 on the generic path)
  *   *ctas_out   total CTAs of the main kernel
  * Any of the three may be NULL.  Host-only; needs no device.
  */
@@ -128,6 +128,14 @@ int more_route_status(void* stream);
 
 /* more_route_launches -- number of kernels this library has launched in this process (all devices). */
 long long more_route_launches(void);
+
+/*
+ * more_route_debug_counters -- diagnostic.  Synchronise `stream`, copy the current device's 16 epilogue event
+ * counters to out16 (host) and clear them.  The kernels only maintain the counters when the library was built
+ * with -DMORE_STATS (chunks, chunks with a hit, triples with a hit, appended candidates, list refreshes, refresh
+ * iterations, rescans, element-by-element chunks; the rest unused); otherwise they read zero.
+ */
+int more_route_debug_counters(unsigned long long* out16, void* stream);
 
 /* more_strerror -- a static, human-readable string for a MORE_* code. */
 const char* more_strerror(int code);

@@ -30,12 +30,13 @@ struct DeviceCtx {
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
     int* status = nullptr;        // device int: 0 = ok, else a MORE_ERR_* code written by a kernel
+    unsigned long long* stats = nullptr;   // 16 diagnostic counters, next to the status word
     void* staging = nullptr;      // device staging of more_route_host
     size_t staging_bytes = 0;
 };
 
 // Tokens per CTA of the tensor-core path, and the expert-tile width of one accumulator buffer.
-constexpr int kBlockTokens = 128;
+constexpr int kBlockTokens = 256;
 constexpr int kTileExperts = 128;
 
 // Launch plan (host-only logic, testable without a device).

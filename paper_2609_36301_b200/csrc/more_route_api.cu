@@ -26,8 +26,11 @@ int get_ctx(DeviceCtx** out)
         c.cc_major = major;
         c.sm_count = sms;
         if (major != 10) return MORE_ERR_ARCH;
-        if (cudaMalloc(&c.status, sizeof(int)) != cudaSuccess) return MORE_ERR_CUDA;
-        if (cudaMemset(c.status, 0, sizeof(int)) != cudaSuccess) return MORE_ERR_CUDA;
+        void* blk = nullptr;                   // status word + 16 diagnostic counters
+        if (cudaMalloc(&blk, 256) != cudaSuccess) return MORE_ERR_CUDA;
+        if (cudaMemset(blk, 0, 256) != cudaSuccess) return MORE_ERR_CUDA;
+        c.status = static_cast<int*>(blk);
+        c.stats = reinterpret_cast<unsigned long long*>(static_cast<char*>(blk) + 128);
         c.dev = dev;
     }
     if (c.cc_major != 10) return MORE_ERR_ARCH;
@@ -235,6 +238,19 @@ int more_route_status(void* stream)
 }
 
 long long more_route_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int more_route_debug_counters(unsigned long long* out16, void* stream)
+{
+    if (!out16) return MORE_ERR_NULL;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(out16, ctx->stats, 16 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MORE_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->stats, 0, 16 * sizeof(unsigned long long), st) != cudaSuccess) return MORE_ERR_CUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
 
 const char* more_strerror(int code)
 {

@@ -96,7 +96,7 @@ __global__ void generic_route_tokens(const float* __restrict__ Z, const __nv_bfl
         out_idx[n * k + lane] = li;
         out_gate[n * k + lane] = g;
         if (out_topval) out_topval[n * k + lane] = lv;
-        atomicAdd(out_counts + li, 1);
+        if ((unsigned)li < (unsigned)M) atomicAdd(out_counts + li, 1);   // (non-finite inputs can leave a slot unfilled)
     }
     if (out_lse && lane == 0) out_lse[n] = m_all + logf(z_all);
 }

@@ -2,25 +2,27 @@
 // accumulators, a thread-per-token epilogue that keeps the running top-k (and, on request, the online
 // (max, sum-of-exponentials) pair of Eq. app_online) in registers.
 //
-// One CTA routes one block of 128 tokens over one contiguous range of expert tiles (Algorithm 1, with the token
-// block additionally split over `msplit` CTAs along the expert dimension):
+// One CTA routes one block of 256 tokens (two 128-row accumulators) over one contiguous range of expert tiles
+// (Algorithm 1, with the token block additionally split over `msplit` CTAs along the expert dimension):
 //
-//   phase 1  z = X_blk R1            TMA streams 128x64 X tiles and 64x64 R1 tiles (zero-filled beyond r),
-//                                    tcgen05.mma accumulates the 128 x 64 fp32 block in TMEM.
-//   narrow   z -> bf16 hi + bf16 lo  written to shared memory as the K-major A operand [hi | lo].  Carrying both
+//   phase 1  z = X_blk R1            TMA streams 256x64 X tiles and 64x64 R1 tiles (zero-filled beyond r),
+//                                    tcgen05.mma accumulates two 128 x 64 fp32 blocks in TMEM.
+//   narrow   z -> bf16 hi + bf16 lo  written to shared memory as the K-major A operands [hi | lo].  Carrying both
 //                                    parts keeps the logits within ~3e-5 of exact arithmetic.
-//   phase 2  y = z R2[:, tile]       one 128-expert tile at a time: TMA brings the r x 128 slice of R2, tcgen05.mma
-//                                    (hi then lo into the same accumulator) fills one of two TMEM buffers while
-//                                    the epilogue drains the other: TMEM lane = token, so each epilogue thread owns
-//                                    one token and reads its logits 32 columns at a time.
-//   merge    running top-k           sorted (value, id) list in registers; a chunk is looked at element by element
-//                                    only if its maximum beats the list's last entry.
+//   phase 2  y = z R2[:, tile]       one 128-expert tile at a time: TMA brings the r x 128 slice of R2 once for
+//                                    both accumulators (this halves the L2 traffic of re-reading R2 per token
+//                                    block), tcgen05.mma (hi then lo into the same accumulator) fills TMEM,
+//                                    the epilogue drains it: TMEM lane = token, so each epilogue thread owns one
+//                                    token and reads its logits 32 columns at a time.
+//   merge    running top-k           sorted (value, id) list in registers, fed through a small per-token candidate
+//                                    buffer in shared memory (see Selector).
 //   finish   gates, ids, counts      written by the CTA itself (msplit == 1) or, after the partial lists have been
 //                                    parked in scratch, by whichever CTA of the token block finishes last.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..5 = epilogue (warp w reads
-// TMEM lanes 32*(w%4)..).  Two CTAs are resident per SM (256 TMEM columns and ~100 KB of shared memory each), so
-// one CTA's HBM-bound phase 1 overlaps the other's expert sweep.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..9 = epilogue (warp w reads
+// TMEM lanes 32*(w%4).. of accumulator (w-2)/4).  Two CTAs are resident per SM (256 TMEM columns and ~112 KB of
+// shared memory each): while one CTA's epilogue drains its accumulators the other CTA's MMAs run, and one CTA's
+// HBM-bound phase 1 overlaps the other's expert sweep.
 //
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
 // status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
@@ -33,15 +35,16 @@ namespace more {
 
 namespace {
 
-constexpr int kThreads = 192;
-constexpr int kEpilogueThreads = 128;
-constexpr int kStagesP1 = 4;                       // phase-1 ring: 16 KB of X + 8 KB of R1 per stage
-constexpr int kXTileBytes = kBlockTokens * 128;    // 128 tokens x 64 bf16
+constexpr int kThreads = 320;                      // warps 0, 1: TMA / MMA; warps 2..9: epilogue
+constexpr int kEpilogueThreads = 256;              // one thread per token of the block
+constexpr int kStagesP1 = 2;                       // phase-1 ring: 32 KB of X + 8 KB of R1 per stage
+constexpr int kXTileBytes = kBlockTokens * 128;    // 256 tokens x 64 bf16
 constexpr int kR1TileBytes = 64 * 128;             // 64 K-rows x 64 bf16 (columns >= r are zero-filled by TMA)
 constexpr int kP1StageBytes = kXTileBytes + kR1TileBytes;
-constexpr int kRingBytes = kStagesP1 * kP1StageBytes;   // 96 KB, reused by phase 2
+constexpr int kRingBytes = 110 * 1024;             // phase 1: the two stages; phase 2: A operands, candidates, R2 stages
+static_assert(kStagesP1 * kP1StageBytes <= kRingBytes, "phase-1 ring does not fit");
 constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
-constexpr int kTmemCols = 256;                     // two 128-column fp32 accumulator buffers
+constexpr int kTmemCols = 256;                     // two 128-token x 128-expert fp32 accumulators
 constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers
@@ -79,6 +82,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+        __nanosleep(32);
         if ((++spins & 255u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitBudgetCycles) {
@@ -230,33 +234,50 @@ struct TopList {
         v[0] = top ? x : v[0];
         id[0] = top ? j : id[0];
     }
+    // Insert with the full order (value descending, id ascending): for merging lists whose ids interleave.
+    __device__ __forceinline__ void insert_ordered(float x, int j)
+    {
+        auto ahead = [&](int s) { return x > v[s] || (x == v[s] && j < id[s]); };
+#pragma unroll
+        for (int s = KCAP - 1; s > 0; --s) {
+            const bool above_prev = ahead(s - 1);
+            const bool above_this = ahead(s);
+            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
+            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
+        }
+        const bool top = ahead(0);
+        v[0] = top ? x : v[0];
+        id[0] = top ? j : id[0];
+    }
 };
 
 // Running top-k of one token.  Between refreshes the sorted list is left alone: elements that beat the cached
 // threshold `tau` (the list's last entry as of the last refresh) are only appended, in ascending column order, to
 // this thread's column of a shared-memory candidate buffer (one predicated 8-byte store each); refresh() then
-// inserts them one by one.  Control flow around the appends is warp-uniform (votes), so the 32 tokens of a warp
-// never serialise on one another's hits, and the inserts of several chunks are executed together.
-constexpr int kCandCap = 16;                              // candidate slots per token
-constexpr int kCandSlotStride = kBlockTokens * 8;         // bytes between successive slots of one token
-constexpr int kCandBytes = kCandCap * kCandSlotStride;
-constexpr int kRefreshAt = 2;                             // refresh a warp after a tile once some token holds this many
+// inserts them one by one, so the inserts of several chunks of all 32 tokens of a warp are executed together.
+constexpr int kCandSlotStride = kEpilogueThreads * 8;     // bytes between successive slots of one thread
+#ifndef MORE_WARN
+#define MORE_WARN 2
+#endif
+constexpr int kRefreshAt = MORE_WARN;                     // a warp folds its buffers once some token holds this many
 constexpr unsigned kFullMask = 0xffffffffu;
 
-template <int KCAP>
+template <int KCAP, int CAP>
 struct Selector {
     TopList<KCAP> L;
     float tau;
     uint32_t ptr;     // shared-memory address of this thread's next free candidate slot
     uint32_t base;    // its first slot
     uint32_t lim;     // ptr is clamped here after every triple; reaching it means "may have lost candidates"
+    uint32_t warn;    // at or beyond this fill level the warp refreshes after the chunk
 
     __device__ __forceinline__ void init(uint32_t first_slot)
     {
         L.init();
         tau = -INFINITY;
         base = ptr = first_slot;
-        lim = first_slot + (kCandCap - 3) * kCandSlotStride;
+        lim = first_slot + (CAP - 3) * kCandSlotStride;
+        warn = first_slot + (kRefreshAt < CAP - 3 ? kRefreshAt : CAP - 3) * kCandSlotStride;
     }
     __device__ __forceinline__ void refresh()
     {
@@ -282,14 +303,13 @@ struct Selector {
             : "memory");
     }
     // v: 32 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]); t[10] covers v[30], v[31].
-    // Called by all 32 lanes.  Every element above tau is appended, or, if some token's buffer could not take
-    // them all, the whole warp folds its buffers into the lists and inserts this chunk's elements directly.
+    // Appends every element above tau; if the buffer cannot take them all, ptr ends at lim (the caller then redoes
+    // the chunk element by element).
     __device__ __forceinline__ void scan(const float (&v)[32], const float (&t)[11], int col0)
     {
-        const uint32_t mark = ptr;
 #pragma unroll
         for (int i = 0; i < 11; ++i) {
-            if (__any_sync(kFullMask, t[i] > tau)) {
+            if (t[i] > tau) {
 #pragma unroll
                 for (int e = 0; e < 3; ++e) {
                     const int pos = 3 * i + e;
@@ -297,14 +317,6 @@ struct Selector {
                 }
                 ptr = min(ptr, lim);
             }
-        }
-        if (__any_sync(kFullMask, ptr >= lim)) {
-            ptr = mark;                      // forget this chunk's appends (all tokens of the warp) ...
-            refresh();                       // ... fold the older candidates into the lists ...
-#pragma unroll
-            for (int i = 0; i < 32; ++i)     // ... and take this chunk element by element
-                if (v[i] > L.tau()) L.insert(v[i], col0 + i);
-            tau = L.tau();
         }
     }
 };
@@ -318,6 +330,7 @@ struct KernelParams {
     float* out_topval;
     float* out_lse;
     int* status;
+    unsigned long long* stats;   // diagnostic event counters (only written by -DMORE_STATS builds)
     // scratch (msplit > 1): per token block an arrival counter, per (token, split) a partial list and (m, Z)
     unsigned* counters;
     float* part_val;
@@ -348,7 +361,7 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
             p.out_idx[row * k + q] = L.id[q];
             p.out_gate[row * k + q] = ex2f(L.v[q] * kLog2e - ref2) * inv;
             if (p.out_topval) p.out_topval[row * k + q] = L.v[q];
-            atomicAdd(p.out_counts + L.id[q], 1);
+            if ((unsigned)L.id[q] < (unsigned)p.M) atomicAdd(p.out_counts + L.id[q], 1);   // (non-finite inputs can leave a slot unfilled)
         }
     }
     if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
@@ -360,12 +373,14 @@ __global__ void __launch_bounds__(kThreads, 2)
 route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
                      const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
 {
-    constexpr int kKSteps = RPAD / 16;                       // UMMA K = 16
-    constexpr int kZopBytes = (RPAD == 64) ? 32768 : 16384;  // [hi | lo] rows of 128 B; two slabs when 2*RPAD > 64
-    constexpr int kR2StageBytes = RPAD * 256;                // two 64-expert blocks of RPAD rows x 128 B
-    constexpr int kP2Free = kRingBytes - kZopBytes - kCandBytes;
-    constexpr int kStagesP2 = (kP2Free / kR2StageBytes) > 8 ? 8 : (kP2Free / kR2StageBytes);
-    static_assert(kStagesP2 >= 2, "R2 ring needs at least two stages");
+    constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
+    constexpr int kZopOne = (RPAD == 64) ? 32768 : 16384;       // A operand [hi | lo] of one 128-token accumulator
+    constexpr int kZopBytes = 2 * kZopOne;
+    constexpr int kR2StageBytes = RPAD * 256;                   // one 128-expert tile: two 64-expert blocks of RPAD rows x 128 B
+    constexpr int kStagesP2 = (RPAD == 64) ? 2 : 4;             // tiles in flight
+    constexpr int kCandCap = (RPAD == 64) ? 7 : 16;             // candidate slots per token (what the ring has room for)
+    constexpr int kCandBytes = kCandCap * kCandSlotStride;
+    static_assert(kZopBytes + kCandBytes + kStagesP2 * kR2StageBytes <= kRingBytes, "phase-2 layout does not fit");
     constexpr float kLog2e = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
@@ -376,8 +391,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
     // barrier slots
     constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kStagesP1, B_ZACC = B_EMPTY1 + kStagesP1, B_ZOP = B_ZACC + 1,
-                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
-                  B_COUNT = B_ACCE + 2;
+                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 1,
+                  B_COUNT = B_ACCE + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
@@ -398,7 +413,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         mbar_init(bar(B_ZACC), 1);
         mbar_init(bar(B_ZOP), kEpilogueThreads);
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads); }
+        mbar_init(bar(B_ACCF), 1);
+        mbar_init(bar(B_ACCE), kEpilogueThreads);
         *abort_flag = 0;
         *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -413,8 +429,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t zop = ring;                        // phase 2: A operand [hi | lo]
-    const uint32_t r2ring = ring + kZopBytes + kCandBytes;   // phase 2: R2 stages (after the candidate buffers)
+    const uint32_t zop = ring;                                  // phase 2: A operands, accumulator 0 then 1
+    const uint32_t cand = ring + kZopBytes;                     // phase 2: candidate buffers
+    const uint32_t r2ring = ring + kZopBytes + kCandBytes;      // phase 2: R2 stages
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
@@ -426,7 +443,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 if (!ok) break;
                 const uint32_t dst = ring + s * kP1StageBytes;
                 mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
-                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);
+                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // 256 token rows x 64 columns
                 tma_load_2d(dst + kXTileBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
             }
             // the ring is reused by phase 2: wait until every phase-1 MMA has finished reading it
@@ -455,10 +472,13 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 tc_fence_after();
                 const uint32_t xa = ring + s * kP1StageBytes, rb = xa + kXTileBytes;
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t ad = umma_desc_sw128(xa + kk * 32, 16, 1024);            // K-major, +32 B per K=16
-                    const uint64_t bd = umma_desc_sw128(rb + kk * 2048, 8192, 1024);        // MN-major, 16 K-rows
-                    tc_mma_bf16(tmem_base, ad, bd, idesc1, (kt | kk) != 0);
+                for (int a = 0; a < 2; ++a) {
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        const uint64_t ad = umma_desc_sw128(xa + a * 16384 + kk * 32, 16, 1024);   // K-major, +32 B per K=16
+                        const uint64_t bd = umma_desc_sw128(rb + kk * 2048, 8192, 1024);           // MN-major, 16 K-rows
+                        tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc1, (kt | kk) != 0);
+                    }
                 }
                 tc_commit(bar(B_EMPTY1 + s));
             }
@@ -466,34 +486,40 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             ok = ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status);
             tc_fence_after();
             for (int it = 0; it < ntiles && ok; ++it) {
-                const int s = it % kStagesP2, b = it & 1;
+                const int s = it % kStagesP2;
                 ok = mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status);
-                ok = ok && mbar_wait(bar(B_ACCE + b), ((it >> 1) & 1) ^ 1, abort_flag, p.status);
+                ok = ok && mbar_wait(bar(B_ACCE), (it & 1) ^ 1, abort_flag, p.status);    // previous tile drained
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t rb = r2ring + s * kR2StageBytes;
 #pragma unroll
-                for (int j = 0; j < 2 * kKSteps; ++j) {
-                    const uint32_t abyte = j * 32;                                           // K offset in [hi | lo]
-                    const uint64_t ad = umma_desc_sw128(zop + (abyte >> 7) * 16384 + (abyte & 127), 16, 1024);
-                    const uint64_t bd = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
-                    tc_mma_bf16(tmem_base + b * kTileExperts, ad, bd, idesc2, j != 0);
+                for (int a = 0; a < 2; ++a) {
+#pragma unroll
+                    for (int j = 0; j < 2 * kKSteps; ++j) {
+                        const uint32_t abyte = j * 32;                                       // K offset in [hi | lo]
+                        const uint64_t ad =
+                            umma_desc_sw128(zop + a * kZopOne + (abyte >> 7) * 16384 + (abyte & 127), 16, 1024);
+                        const uint64_t bd = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
+                        tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc2, j != 0);
+                    }
                 }
                 tc_commit(bar(B_EMPTY2 + s));
-                tc_commit(bar(B_ACCF + b));
+                tc_commit(bar(B_ACCF));
             }
         }
     } else {
         // ========================================================================================= epilogue
         const int q = warp & 3;                              // TMEM lane group this warp may read
-        const int row_in_blk = q * 32 + lane;
+        const int acc = (warp - 2) >> 2;                     // which 128-token accumulator
+        const int row_in_acc = q * 32 + lane;
+        const int row_in_blk = acc * 128 + row_in_acc;
         const int64_t row = (int64_t)tok0 + row_in_blk;
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileExperts;
         bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
         if (ok) {
             // ---- narrow z to [hi | lo] and store it as the K-major, 128-B-swizzled A operand
             tc_fence_after();
-            uint8_t* zrow = ring_ptr + row_in_blk * 128;
+            uint8_t* zrow = ring_ptr + acc * kZopOne + row_in_acc * 128;
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
@@ -515,8 +541,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     const int slab_hi = ch_hi >> 3, slab_lo = ch_lo >> 3;
                     uint4 vh = make_uint4(hi[half * 4], hi[half * 4 + 1], hi[half * 4 + 2], hi[half * 4 + 3]);
                     uint4 vl = make_uint4(lo[half * 4], lo[half * 4 + 1], lo[half * 4 + 2], lo[half * 4 + 3]);
-                    *reinterpret_cast<uint4*>(zrow + slab_hi * 16384 + (((ch_hi & 7) ^ (row_in_blk & 7)) << 4)) = vh;
-                    *reinterpret_cast<uint4*>(zrow + slab_lo * 16384 + (((ch_lo & 7) ^ (row_in_blk & 7)) << 4)) = vl;
+                    *reinterpret_cast<uint4*>(zrow + slab_hi * 16384 + (((ch_hi & 7) ^ (row_in_acc & 7)) << 4)) = vh;
+                    *reinterpret_cast<uint4*>(zrow + slab_lo * 16384 + (((ch_lo & 7) ^ (row_in_acc & 7)) << 4)) = vl;
                 }
             }
             fence_async_smem();
@@ -524,83 +550,114 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             mbar_arrive(bar(B_ZOP));
         }
 
-        Selector<KCAP> S;
-        S.init(ring + kZopBytes + row_in_blk * 8);
+        Selector<KCAP, kCandCap> S;
+        S.init(cand + row_in_blk * 8);
+#ifdef MORE_STATS
+        unsigned st_chunks = 0, st_hit = 0, st_trip = 0, st_app = 0, st_rcall = 0, st_riter = 0, st_retry = 0, st_direct = 0;
+#define STAT(x) x
+#else
+#define STAT(x)
+#endif
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
 
-        // One 32-column chunk: triple maxima, optional online softmax update, candidate scan.
-        auto process = [&](float (&v)[32], int col0, bool ragged) {
-            if (ragged) {
-#pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    if (col0 + i >= p.M) v[i] = -INFINITY;
-            }
-            float t[11];
-#pragma unroll
-            for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-            t[10] = fmaxf(v[30], v[31]);
-            const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
-            const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
-            if (LSE) {
-                const float c2 = cmax * kLog2e;
-                if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
-                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; i += 4) {
-                    a0 += ex2f(fmaf(v[i], kLog2e, -m2));
-                    a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
-                    a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
-                    a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
-                }
-                zsum += (a0 + a1) + (a2 + a3);
-            }
-            if (__any_sync(kFullMask, cmax > S.tau)) S.scan(v, t, col0);
-        };
-
-        // `ok` is kept warp-uniform from here on (the votes above need all 32 lanes).
+        // `ok` is kept warp-uniform from here on (tcgen05.ld and the votes below need all 32 lanes).
         ok = __all_sync(kFullMask, ok);
-        float va[32], vb[32];
-        if (ok && ntiles > 0) {
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + 0), 0, abort_flag, p.status));
-            if (ok) {
-                tc_fence_after();
-                tmem_ld32(t_lane, va);
-            }
-        }
         for (int it = 0; it < ntiles && ok; ++it) {
-            const int b = it & 1;
-            const uint32_t tb = t_lane + b * kTileExperts;
             const int e0 = (tile_lo + it) * kTileExperts;
             const bool ragged = e0 + kTileExperts > p.M;
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF), it & 1, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
 #pragma unroll 1
-            for (int half = 0; half < 2; ++half) {
-                tmem_ld_wait32(va);
-                tmem_ld32(tb + half * 64 + 32, vb);
-                process(va, e0 + half * 64, ragged);
-                tmem_ld_wait32(vb);
-                if (half == 0) {
-                    tmem_ld32(tb + 64, va);
-                } else {
-                    tc_fence_before();
-                    mbar_arrive(bar(B_ACCE + b));            // this accumulator buffer may be overwritten now
-                    if (it + 1 < ntiles) {                   // start on the next tile before finishing this one
-                        ok = __all_sync(kFullMask,
-                                        mbar_wait(bar(B_ACCF + (b ^ 1)), ((it + 1) >> 1) & 1, abort_flag, p.status));
-                        if (ok) {
-                            tc_fence_after();
-                            tmem_ld32(t_lane + (b ^ 1) * kTileExperts, va);
+            for (int c = 0; c < kTileExperts / 32; ++c) {
+                // ---- one 32-column chunk: triple maxima, optional online softmax update, candidate scan
+                const uint32_t ta = t_lane + c * 32;
+                const int col0 = e0 + c * 32;
+                float v[32];
+                tmem_ld32(ta, v);
+                tmem_ld_wait32(v);
+                if (ragged) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i)
+                        if (col0 + i >= p.M) v[i] = -INFINITY;
+                }
+                float t[11];
+#pragma unroll
+                for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+                t[10] = fmaxf(v[30], v[31]);
+                const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
+                const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
+                if (LSE) {
+                    const float c2 = cmax * kLog2e;
+                    if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
+                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                    for (int i = 0; i < 32; i += 4) {
+                        a0 += ex2f(fmaf(v[i], kLog2e, -m2));
+                        a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
+                        a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
+                        a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+                    }
+                    zsum += (a0 + a1) + (a2 + a3);
+                }
+                // Append this chunk's candidates.  When some token of the warp runs out of buffer (always so on the
+                // very first chunk, when tau is -inf) the warp forgets the chunk's appends, folds the older candidates
+                // into the lists and takes the chunk element by element, re-read from tensor memory.
+                STAT(st_chunks++; if (__any_sync(kFullMask, cmax > S.tau)) st_hit++;
+                     for (int i = 0; i < 11; ++i) if (__any_sync(kFullMask, t[i] > S.tau)) st_trip++;)
+                const uint32_t mark = S.ptr;
+                if (cmax > S.tau) S.scan(v, t, col0);
+                STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandSlotStride);)
+                if (__any_sync(kFullMask, S.ptr >= S.lim)) {
+                    S.ptr = mark;
+                    STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
+                    S.refresh();
+#pragma unroll 1
+                    for (int g = 0; g < 4; ++g) {
+                        uint32_t xb[8];
+                        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                                     : "=r"(xb[0]), "=r"(xb[1]), "=r"(xb[2]), "=r"(xb[3]), "=r"(xb[4]), "=r"(xb[5]),
+                                       "=r"(xb[6]), "=r"(xb[7])
+                                     : "r"(ta + g * 8)
+                                     : "memory");
+                        asm volatile("tcgen05.wait::ld.sync.aligned;"
+                                     : "+r"(xb[0]), "+r"(xb[1]), "+r"(xb[2]), "+r"(xb[3]), "+r"(xb[4]), "+r"(xb[5]),
+                                       "+r"(xb[6]), "+r"(xb[7])::"memory");
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const float x = __uint_as_float(xb[i]);
+                            const int cj = col0 + g * 8 + i;
+                            if (cj < p.M && x > S.L.tau()) S.L.insert(x, cj);
                         }
                     }
+                    S.tau = S.L.tau();
+                    STAT(st_direct++;)
                 }
-                process(vb, e0 + half * 64 + 32, ragged);
             }
-            if (__any_sync(kFullMask, S.ptr >= S.base + kRefreshAt * kCandSlotStride)) S.refresh();
+            tc_fence_before();
+            mbar_arrive(bar(B_ACCE));                        // the accumulators may be overwritten now
+            if (__any_sync(kFullMask, S.ptr >= S.warn)) {
+                STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
+                S.refresh();
+            }
         }
         S.refresh();
         TopList<KCAP>& L = S.L;
+#ifdef MORE_STATS
+        if (lane == 0 && p.stats) {
+            atomicAdd(p.stats + 0, (unsigned long long)st_chunks);
+            atomicAdd(p.stats + 1, (unsigned long long)st_hit);
+            atomicAdd(p.stats + 2, (unsigned long long)st_trip);
+            atomicAdd(p.stats + 3, (unsigned long long)st_app);
+            atomicAdd(p.stats + 4, (unsigned long long)st_rcall);
+            atomicAdd(p.stats + 5, (unsigned long long)st_riter);
+            atomicAdd(p.stats + 6, (unsigned long long)st_retry);
+            atomicAdd(p.stats + 7, (unsigned long long)st_direct);
+        }
+#endif
 
-        // ---- finish.  All 128 epilogue threads meet here, also after an abort, so the decision is uniform.
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        // ---- finish.  All 256 epilogue threads meet here, also after an abort, so the decision is uniform.
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abort_flag == 0) {
             if (p.msplit == 1) {
                 if (row < p.T) write_token<KCAP>(p, row, L, m2, zsum);
@@ -614,12 +671,12 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 }
                 p.part_mz[slot] = make_float2(m2, zsum);
                 __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (threadIdx.x == 64) {
                     const unsigned prev = atomicAdd(p.counters + blk, 1u);
                     *last_flag = (prev == (unsigned)p.msplit - 1u);
                 }
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                asm volatile("bar.sync 1, 256;" ::: "memory");
                 if (*last_flag) {
                     __threadfence();
                     const int64_t base = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit;
@@ -746,6 +803,9 @@ int launch_kcap(int k, bool lse, const CUtensorMap& mx, const CUtensorMap& m1, c
                 const KernelParams& kp, int ctas, cudaStream_t st)
 {
     if (k <= 8) return launch_lse<RPAD, 8>(lse, mx, m1, m2, kp, ctas, st);
+#ifdef MORE_ONLY_K8
+    return MORE_ERR_SHAPE;
+#endif
     if (k <= 16) return launch_lse<RPAD, 16>(lse, mx, m1, m2, kp, ctas, st);
     return launch_lse<RPAD, 32>(lse, mx, m1, m2, kp, ctas, st);
 }
@@ -784,6 +844,7 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
     kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
     kp.status = ctx.status;
+    kp.stats = ctx.stats;
     kp.counters = nullptr; kp.part_val = nullptr; kp.part_id = nullptr; kp.part_mz = nullptr;
     if (p.msplit > 1) {
         const size_t blocks = (size_t)(a.T + kBlockTokens - 1) / kBlockTokens;
