@@ -46,6 +46,7 @@ static_assert(kStagesP1 * kP1StageBytes <= kRingBytes, "phase-1 ring does not fi
 constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
 constexpr int kTmemCols = 256;                     // two 128-token x 128-expert fp32 accumulators
 constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s
+constexpr uint32_t kSuspendHintNs = 20000;              // a waiting thread may be parked this long per try
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -67,10 +68,10 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"   // may suspend up to the hinted time
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kSuspendHintNs)
         : "memory");
     return ok;
 }
@@ -82,8 +83,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        __nanosleep(32);
-        if ((++spins & 255u) == 0) {
+        if ((++spins & 15u) == 0) {
             if (*abort_flag) return false;
             if (clock64() - t0 > kWaitBudgetCycles) {
                 *abort_flag = 1;
@@ -302,22 +302,21 @@ struct Selector {
             : "f"(x), "r"(col), "f"(tau), "n"(kCandSlotStride)
             : "memory");
     }
-    // v: 32 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]); t[10] covers v[30], v[31].
-    // Appends every element above tau; if the buffer cannot take them all, ptr ends at lim (the caller then redoes
-    // the chunk element by element).
-    __device__ __forceinline__ void scan(const float (&v)[32], const float (&t)[11], int col0)
+    // v: 16 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]) for i < 5; v[15] stands
+    // alone.  Appends every element above tau; if the buffer cannot take them all, ptr ends at lim (the caller then
+    // redoes the chunk).
+    __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[5], int col0)
     {
 #pragma unroll
-        for (int i = 0; i < 11; ++i) {
+        for (int i = 0; i < 5; ++i) {
             if (t[i] > tau) {
 #pragma unroll
-                for (int e = 0; e < 3; ++e) {
-                    const int pos = 3 * i + e;
-                    if (pos < 32) append_if_above(v[pos], col0 + pos);
-                }
+                for (int e = 0; e < 3; ++e) append_if_above(v[3 * i + e], col0 + 3 * i + e);
                 ptr = min(ptr, lim);
             }
         }
+        append_if_above(v[15], col0 + 15);
+        ptr = min(ptr, lim);
     }
 };
 
@@ -391,8 +390,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
     // barrier slots
     constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kStagesP1, B_ZACC = B_EMPTY1 + kStagesP1, B_ZOP = B_ZACC + 1,
-                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 1,
-                  B_COUNT = B_ACCE + 1;
+                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
+                  B_COUNT = B_ACCE + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
@@ -413,8 +412,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         mbar_init(bar(B_ZACC), 1);
         mbar_init(bar(B_ZOP), kEpilogueThreads);
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
-        mbar_init(bar(B_ACCF), 1);
-        mbar_init(bar(B_ACCE), kEpilogueThreads);
+        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads / 2); }
         *abort_flag = 0;
         *last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -488,12 +486,14 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             for (int it = 0; it < ntiles && ok; ++it) {
                 const int s = it % kStagesP2;
                 ok = mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status);
-                ok = ok && mbar_wait(bar(B_ACCE), (it & 1) ^ 1, abort_flag, p.status);    // previous tile drained
                 if (!ok) break;
-                tc_fence_after();
                 const uint32_t rb = r2ring + s * kR2StageBytes;
 #pragma unroll
                 for (int a = 0; a < 2; ++a) {
+                    // accumulator a is free once its 128 epilogue threads have drained the previous tile
+                    ok = ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
                     for (int j = 0; j < 2 * kKSteps; ++j) {
                         const uint32_t abyte = j * 32;                                       // K offset in [hi | lo]
@@ -502,9 +502,10 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         const uint64_t bd = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
                         tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc2, j != 0);
                     }
+                    tc_commit(bar(B_ACCF + a));
                 }
+                if (!ok) break;
                 tc_commit(bar(B_EMPTY2 + s));
-                tc_commit(bar(B_ACCF));
             }
         }
     } else {
@@ -565,34 +566,29 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         for (int it = 0; it < ntiles && ok; ++it) {
             const int e0 = (tile_lo + it) * kTileExperts;
             const bool ragged = e0 + kTileExperts > p.M;
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF), it & 1, abort_flag, p.status));
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
             if (!ok) break;
             tc_fence_after();
-#pragma unroll 1
-            for (int c = 0; c < kTileExperts / 32; ++c) {
-                // ---- one 32-column chunk: triple maxima, optional online softmax update, candidate scan
-                const uint32_t ta = t_lane + c * 32;
-                const int col0 = e0 + c * 32;
-                float v[32];
-                tmem_ld32(ta, v);
-                tmem_ld_wait32(v);
+            // The tile is read 16 columns at a time into two register buffers: the load of the next 16 columns is
+            // in flight while the current 16 are processed.
+            float va[16], vb[16];
+            // ---- one 16-column chunk: triple maxima, optional online softmax update, candidate scan
+            auto process = [&](float (&v)[16], uint32_t ta, int col0) {
                 if (ragged) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
+                    for (int i = 0; i < 16; ++i)
                         if (col0 + i >= p.M) v[i] = -INFINITY;
                 }
-                float t[11];
+                float t[5];
 #pragma unroll
-                for (int i = 0; i < 10; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                t[10] = fmaxf(v[30], v[31]);
-                const float u0 = max3(t[0], t[1], t[2]), u1 = max3(t[3], t[4], t[5]), u2 = max3(t[6], t[7], t[8]);
-                const float cmax = max3(max3(u0, u1, u2), t[9], t[10]);
+                for (int i = 0; i < 5; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
+                const float cmax = max3(max3(t[0], t[1], t[2]), max3(t[3], t[4], v[15]), -INFINITY);
                 if (LSE) {
                     const float c2 = cmax * kLog2e;
                     if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
                     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-                    for (int i = 0; i < 32; i += 4) {
+                    for (int i = 0; i < 16; i += 4) {
                         a0 += ex2f(fmaf(v[i], kLog2e, -m2));
                         a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
                         a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
@@ -601,19 +597,30 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     zsum += (a0 + a1) + (a2 + a3);
                 }
                 // Append this chunk's candidates.  When some token of the warp runs out of buffer (always so on the
-                // very first chunk, when tau is -inf) the warp forgets the chunk's appends, folds the older candidates
-                // into the lists and takes the chunk element by element, re-read from tensor memory.
+                // very first chunk, when tau is -inf) the warp forgets the chunk's appends and folds the older
+                // candidates into the lists; with empty buffers and a fresher tau the chunk usually fits on a second
+                // scan, otherwise it is taken element by element, re-read from tensor memory.
                 STAT(st_chunks++; if (__any_sync(kFullMask, cmax > S.tau)) st_hit++;
-                     for (int i = 0; i < 11; ++i) if (__any_sync(kFullMask, t[i] > S.tau)) st_trip++;)
+                     for (int i = 0; i < 5; ++i) if (__any_sync(kFullMask, t[i] > S.tau)) st_trip++;)
                 const uint32_t mark = S.ptr;
                 if (cmax > S.tau) S.scan(v, t, col0);
                 STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandSlotStride);)
-                if (__any_sync(kFullMask, S.ptr >= S.lim)) {
+                bool direct = __any_sync(kFullMask, S.ptr >= S.lim);
+                if (direct) {
                     S.ptr = mark;
                     STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
+                    const bool had_older = __any_sync(kFullMask, mark != S.base);
                     S.refresh();
+                    if (had_older) {
+                        STAT(st_retry++;)
+                        if (cmax > S.tau) S.scan(v, t, col0);
+                        direct = __any_sync(kFullMask, S.ptr >= S.lim);
+                        if (direct) S.ptr = S.base;
+                    }
+                }
+                if (direct) {
 #pragma unroll 1
-                    for (int g = 0; g < 4; ++g) {
+                    for (int g = 0; g < 2; ++g) {
                         uint32_t xb[8];
                         asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
                                      : "=r"(xb[0]), "=r"(xb[1]), "=r"(xb[2]), "=r"(xb[3]), "=r"(xb[4]), "=r"(xb[5]),
@@ -633,9 +640,22 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     S.tau = S.L.tau();
                     STAT(st_direct++;)
                 }
+            };
+            tmem_ld16(t_lane, va);
+#pragma unroll 1
+            for (int c = 0; c < kTileExperts / 32; ++c) {
+                const uint32_t ta = t_lane + c * 32;
+                const int col0 = e0 + c * 32;
+                tmem_ld_wait16(va);
+                tmem_ld16(ta + 16, vb);
+                process(va, ta, col0);
+                // (a direct-mode re-read inside process waits for all loads, including the one just issued: harmless)
+                tmem_ld_wait16(vb);
+                if (c + 1 < kTileExperts / 32) tmem_ld16(ta + 32, va);
+                process(vb, ta + 16, col0 + 16);
             }
             tc_fence_before();
-            mbar_arrive(bar(B_ACCE));                        // the accumulators may be overwritten now
+            mbar_arrive(bar(B_ACCE + acc));                  // this accumulator may be overwritten now
             if (__any_sync(kFullMask, S.ptr >= S.warn)) {
                 STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
                 S.refresh();
