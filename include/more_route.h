@@ -110,6 +110,33 @@ int more_route_host(const void* X_host, const void* R1_host, const void* R2_host
                     int32_t* out_idx_host, float* out_gate_host, int32_t* out_counts_host, void* stream);
 
 /*
+ * more_route_noalloc -- more_route for callers that must not allocate device memory.  (The paper has no counterpart;
+ * this is a property of the library, not of the method.)
+ *
+ * Who needs it: a process whose device memory is owned by its own pool and that may not call the CUDA allocator; code
+ * for which a device allocation is unacceptable because it can synchronise the device and stall unrelated streams;
+ * an environment that denies cudaMalloc outright.  This entry point calls no cudaMalloc, cudaFree or any other
+ * allocating routine, ever.  It runs the generic (CUDA-core) kernels, for any shape they accept, and keeps their
+ * only scratch, z = X R1 in fp32, in a fixed 4 MiB array that is part of the library image: every GPU that loads the
+ * library holds that array until the process exits.
+ *
+ *   Limit      T * r <= more_route_noalloc_capacity() (= 1,048,576); beyond it the call returns MORE_ERR_TOO_LARGE
+ *              and does nothing.
+ *   Set-up     the first call on each device looks up the array's device address (cudaGetSymbolAddress) with that
+ *              device current; make that first call before any stream capture begins.
+ *   Sharing    all calls on a device use the same array, which keeps whatever the last call left in it.  Every call
+ *              overwrites what it reads, and clears out_counts on `stream` itself, so no stale data can leak; but two
+ *              calls whose kernels may overlap on the GPU race on the array and must be serialised by the caller.
+ *   Otherwise  arguments, outputs, ordering, errors and asynchrony exactly as more_route.
+ */
+int more_route_noalloc(const void* X, const void* R1, const void* R2,
+                       int T, int h, int r, int M, int k, int gate_mode,
+                       int32_t* out_idx, float* out_gate, int32_t* out_counts, void* stream);
+
+/* more_route_noalloc_capacity -- the largest T * r more_route_noalloc accepts. */
+long long more_route_noalloc_capacity(void);
+
+/*
  * more_route_plan -- report, without launching, what more_route_ex would do for a shape:
  *   *path_out   MORE_PATH_GENERIC or MORE_PATH_TCGEN05
  *   *msplit_out CTAs per 256-token block (1 on the generic path)

@@ -43,6 +43,10 @@ def lib() -> ctypes.CDLL:
         L.more_route_ex.restype = i32
         L.more_route_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.more_route_host.restype = i32
+        L.more_route_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
+        L.more_route_noalloc.restype = i32
+        L.more_route_noalloc_capacity.argtypes = []
+        L.more_route_noalloc_capacity.restype = ctypes.c_longlong
         ip = ctypes.POINTER(ctypes.c_int)
         L.more_route_plan.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, ip, ip, ip]
         L.more_route_plan.restype = i32
@@ -129,6 +133,22 @@ def more_route_host(X, R1, R2, k, gate_mode, out_idx, out_gate, out_counts, stre
                                hp(out_counts), _stream(stream))
     if rc != 0:
         raise MoreRouteError(rc, "more_route_host")
+
+
+def more_route_noalloc(X, R1, R2, k, gate_mode, out_idx, out_gate, out_counts, stream=None):
+    """``more_route_noalloc`` of the C interface: same arguments as :func:`more_route`; the library allocates nothing
+    (its scratch is a fixed array inside the library image) and rejects ``T * r`` beyond
+    :func:`more_route_noalloc_capacity` with ``MORE_ERR_TOO_LARGE``.  For callers that may not use the CUDA allocator."""
+    T, h = X.shape
+    r, M = R2.shape
+    rc = lib().more_route_noalloc(_ptr(X), _ptr(R1), _ptr(R2), T, h, r, M, k, gate_mode,
+                                  _ptr(out_idx), _ptr(out_gate), _ptr(out_counts), _stream(stream))
+    if rc != 0:
+        raise MoreRouteError(rc, "more_route_noalloc")
+
+
+def more_route_noalloc_capacity() -> int:
+    return int(lib().more_route_noalloc_capacity())
 
 
 def more_route_status(stream=None) -> int:
