@@ -253,6 +253,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-context", action="store_true", help="skip the unfused library-op router (context only)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -355,7 +356,7 @@ def main():
                 clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roof)
 
     # ---- context: unfused library-op router on the same inputs
-    ms_unfused = unfused_reference_ms(torch, bufs, case, gate_mode)
+    ms_unfused = None if args.no_context else unfused_reference_ms(torch, bufs, case, gate_mode)
     line["unfused_gpu_reference_ms"] = ms_unfused
 
     # ---- the CPU oracle on the host cores (a reported baseline, not the target)

@@ -35,7 +35,7 @@ struct DeviceCtx {
     size_t staging_bytes = 0;
 };
 
-// Tokens per CTA of the tensor-core path, and the expert-tile width of one accumulator buffer.
+// Largest number of tokens per CTA of the tensor-core path (rows of one X tile), and the expert-tile width.
 constexpr int kBlockTokens = 256;
 constexpr int kTileExperts = 128;
 
@@ -45,6 +45,7 @@ struct Plan {
     int msplit;   // CTAs per token block
     int ctas;     // CTAs of the main kernel
     int rpad;     // r rounded up to a multiple of 16 (tensor-core path)
+    int block_tokens;   // tokens per CTA (tensor-core path): multiple of 32, <= kBlockTokens
 };
 
 bool tcgen05_shape_ok(int T, int h, int r, int M, int k);

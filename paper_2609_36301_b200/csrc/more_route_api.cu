@@ -104,37 +104,44 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
     p.rpad = (r + 15) / 16 * 16;
     if (path == MORE_PATH_GENERIC || !fast_ok) {
         p.path = MORE_PATH_GENERIC;
+        p.block_tokens = 8;
         p.msplit = 1;
         p.ctas = (T + 7) / 8;
         *out = p;
         return MORE_OK;
     }
     p.path = MORE_PATH_TCGEN05;
-    const int blocks = (T + kBlockTokens - 1) / kBlockTokens;
+    if (sm_count <= 0) sm_count = 148;
+    const int slots = 2 * sm_count;                       // two CTAs are resident per SM
     const int tiles = (M + kTileExperts - 1) / kTileExperts;
-    int s = msplit;
-    if (s == 0) {
-        // Pick the split that minimises (rounds of CTAs over the SMs) x (time of one CTA).  One CTA costs the
-        // z projection (~ h columns of X) plus its share of the expert sweep; weigh a logit column like
-        // `w` X columns (the sweep's per-column cost relative to streaming one X column).
-        if (sm_count <= 0) sm_count = 148;
-        const double w = 1.0;
-        const int slots = 2 * sm_count;                 // two CTAs are resident per SM
-        double best = 1e300;
-        s = 1;
-        for (int c = 1; c <= 64 && c <= tiles; ++c) {
-            const long long ctas = (long long)blocks * c;
-            const double rounds = (double)((ctas + slots - 1) / slots);
-            const double per_cta = 0.25 * h + w * ((tiles + c - 1) / c) * kTileExperts + 512.0;
-            const double cost = rounds * per_cta;
-            if (cost < best * 0.97) { best = cost; s = c; }
+    // Fill one wave of resident CTAs as evenly as possible.  Candidates: tokens per CTA (a multiple of 32 up to
+    // 256; smaller blocks waste rows of the second accumulator but even out the SMs) x CTAs per token block
+    // (each extra CTA repeats the block's z projection and starts its top-k from scratch, and a second, partial
+    // wave costs more than it gains; every CTA keeps at least four expert tiles).
+    double best = 1e300;
+    int best_bt = kBlockTokens, best_s = 1;
+    for (int bt = kBlockTokens; bt >= 128; bt -= 32) {
+        const int blocks = (T + bt - 1) / bt;
+        int s = msplit;
+        if (s == 0) {
+            s = slots / blocks;
+            if (s > tiles / 4) s = tiles / 4;
+            if (s < 1) s = 1;
+            if (s > 64) s = 64;
         }
+        if (s > tiles) s = tiles;
+        const long long ctas = (long long)blocks * s;
+        // makespan ~ (CTAs the busiest SM gets) x (time of one CTA); one CTA costs its projection (the X tile always
+        // has 256 rows), its share of the sweep (proportional to its live token rows) and a start-up term
+        const double per_sm = (double)((ctas + sm_count - 1) / sm_count);
+        const double per_cta = 256.0 * (h / 8.0) + (double)bt * ((double)tiles / s) * 16.0 + 256.0 * 256.0;
+        const double cost = per_sm * per_cta;
+        if (cost < best * 0.999) { best = cost; best_bt = bt; best_s = s; }
     }
-    if (s > tiles) s = tiles;
-    if (s < 1) s = 1;
-    if (s > 64) return MORE_ERR_SHAPE;
-    p.msplit = s;
-    p.ctas = blocks * s;
+    if (best_s > 64) return MORE_ERR_SHAPE;
+    p.block_tokens = best_bt;
+    p.msplit = best_s;
+    p.ctas = ((T + best_bt - 1) / best_bt) * best_s;
     *out = p;
     return MORE_OK;
 }

@@ -307,6 +307,14 @@ struct Selector {
     // redoes the chunk).
     __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[5], int col0)
     {
+#ifdef MORE_FLAT_SCAN
+        (void)t;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+            append_if_above(v[i], col0 + i);
+            if (i % 3 == 2 || i == 15) ptr = min(ptr, lim);
+        }
+#else
 #pragma unroll
         for (int i = 0; i < 5; ++i) {
             if (t[i] > tau) {
@@ -317,11 +325,13 @@ struct Selector {
         }
         append_if_above(v[15], col0 + 15);
         ptr = min(ptr, lim);
+#endif
     }
 };
 
 struct KernelParams {
     int T, h, r, M, k, gate_mode, msplit;
+    int block_tokens;            // tokens routed per CTA: a multiple of 32, at most 256 (the X tile always has 256 rows)
     int tiles_total;             // ceil(M / 128)
     int32_t* out_idx;
     float* out_gate;
@@ -400,7 +410,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int blk = blockIdx.x / p.msplit, split = blockIdx.x % p.msplit;
-    const int tok0 = blk * kBlockTokens;
+    const int tok0 = blk * p.block_tokens;
     // expert tiles of this CTA: an even share of ceil(M/128) tiles
     const int tile_lo = (int)(((long long)p.tiles_total * split) / p.msplit);
     const int tile_hi = (int)(((long long)p.tiles_total * (split + 1)) / p.msplit);
@@ -515,6 +525,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int row_in_acc = q * 32 + lane;
         const int row_in_blk = acc * 128 + row_in_acc;
         const int64_t row = (int64_t)tok0 + row_in_blk;
+        const bool row_live = row_in_blk < p.block_tokens && row < p.T;     // rows past the block belong to the next CTA
+        const bool warp_live = acc * 128 + q * 32 < p.block_tokens;         // warp-uniform: block_tokens is a multiple of 32
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileExperts;
         bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
         if (ok) {
@@ -568,6 +580,10 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const bool ragged = e0 + kTileExperts > p.M;
             ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
             if (!ok) break;
+            if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
+                mbar_arrive(bar(B_ACCE + acc));
+                continue;
+            }
             tc_fence_after();
             // The tile is read 16 columns at a time into two register buffers: the load of the next 16 columns is
             // in flight while the current 16 are processed.
@@ -680,7 +696,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abort_flag == 0) {
             if (p.msplit == 1) {
-                if (row < p.T) write_token<KCAP>(p, row, L, m2, zsum);
+                if (row_live) write_token<KCAP>(p, row, L, m2, zsum);
             } else {
                 // park the partial list; the CTA that arrives last for this token block merges all of them
                 const int64_t slot = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit + split;
@@ -716,7 +732,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                             gm = nm;
                         }
                     }
-                    if (row < p.T) write_token<KCAP>(p, row, G, gm, gz);
+                    if (row_live) write_token<KCAP>(p, row, G, gm, gz);
                     if (threadIdx.x == 64) p.counters[blk] = 0;   // ready for the next call
                 }
             }
@@ -843,7 +859,7 @@ bool tcgen05_shape_ok(int T, int h, int r, int M, int k)
 size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p)
 {
     if (p.msplit <= 1) return 0;
-    const size_t blocks = (size_t)(a.T + kBlockTokens - 1) / kBlockTokens;
+    const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
     const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
     const size_t kc = (size_t)kcap_of(a.k);
     return align_up(blocks * 4, 256) + align_up(slots * kc * 4, 256) * 2 + align_up(slots * 8, 256);
@@ -860,6 +876,7 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
 
     KernelParams kp;
     kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
+    kp.block_tokens = p.block_tokens;
     kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
     kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
     kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
@@ -867,7 +884,7 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     kp.stats = ctx.stats;
     kp.counters = nullptr; kp.part_val = nullptr; kp.part_id = nullptr; kp.part_mz = nullptr;
     if (p.msplit > 1) {
-        const size_t blocks = (size_t)(a.T + kBlockTokens - 1) / kBlockTokens;
+        const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
         const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
         const size_t kc = (size_t)kcap_of(a.k);
         char* base = static_cast<char*>(scratch);

@@ -62,7 +62,9 @@ def test_plan_picks_paths_and_splits():
     with pytest.raises(mr.MoreRouteError):
         P(100, 20, 5, 33, 3, path=mr.PATH_TCGEN05)
     p = P(8192, 4096, 64, 131072, 16)
-    assert p.msplit > 1 and p.ctas == 32 * p.msplit             # few token blocks, many experts: split the experts
+    assert p.msplit > 1 and p.ctas % p.msplit == 0              # few token blocks, many experts: split the experts
+    assert 32 <= p.ctas // p.msplit <= 64 and p.ctas <= 296     # 128..256 tokens per CTA, one wave of 2 CTAs per SM
+    assert P(65536, 2048, 64, 16384, 8).ctas in range(256, 297)
     assert P(32768, 512, 32, 1024, 8).msplit * 128 <= 1024      # never more CTAs per block than expert tiles
     assert P(300, 256, 32, 4096, 8, msplit=5).msplit == 5
     assert P(300, 256, 32, 256, 8, msplit=5).msplit == 2        # clamped to the number of 128-expert tiles
