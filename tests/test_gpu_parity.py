@@ -211,3 +211,49 @@ def test_non_default_stream_and_repeat_calls():
         assert torch.equal(o.gate, outs[0].gate)
     assert mr.more_route_status(s) == 0
     assert mr.launches() > 0
+
+
+def test_k_equals_m_on_tensor_core_path():
+    """Every expert selected (k == M): the list is the whole sorted row."""
+    case = inputs.gaussian_case(200, 64, 16, 16, 16, 1, seed=12)
+    assert mr.more_route_plan(200, 64, 16, 16, 16).path == mr.PATH_TCGEN05
+    idx, gate, counts, topval, lse = run_gpu(case, path=mr.PATH_TCGEN05)
+    assert np.array_equal(np.sort(idx, axis=1), np.broadcast_to(np.arange(16), (200, 16)))
+    assert np.all(counts == 200)
+    np.testing.assert_allclose(gate.sum(axis=1), 1.0, atol=1e-5)       # P over all experts sums to one
+    full_check(case, mr.PATH_TCGEN05, 1)
+
+
+def test_sorted_ascending_logits_worst_case_for_the_running_threshold():
+    """Experts ordered so that every token's logits increase with the expert id: every new column beats the running
+    threshold, the worst case for the candidate buffers (they overflow constantly)."""
+    case = inputs.gaussian_case(256, 64, 8, 1024, 8, 0, seed=13)
+    # make all logits of a token increase with the expert id: z has one positive component, R2 is a ramp
+    R1f = np.zeros((64, 8), dtype=np.float32); R1f[0, 0] = 1.0
+    Xf = inputs.bf16_bits_to_f32(case.X); Xf[:, 0] = np.abs(Xf[:, 0]) + 0.5
+    R2f = np.zeros((8, 1024), dtype=np.float32); R2f[0] = np.arange(1024, dtype=np.float32) / 128.0
+    case.X, case.R1, case.R2 = inputs.to_bf16_bits(Xf), inputs.to_bf16_bits(R1f), inputs.to_bf16_bits(R2f)
+    for path in (mr.PATH_TCGEN05, mr.PATH_GENERIC):
+        idx, *_ = run_gpu(case, path=path)
+        ref = oracle.route(case.X, case.R1, case.R2, 8, 0)
+        assert np.array_equal(idx, ref.idx)            # bf16 ramp has exact ties: ids ascending within ties
+
+
+def test_non_finite_inputs_terminate_and_leave_other_tokens_alone():
+    import torch
+    case = inputs.gaussian_case(300, 64, 16, 512, 4, 1, seed=14)
+    Xf = inputs.bf16_bits_to_f32(case.X)
+    Xf[7, :] = np.nan
+    Xf[130, 3] = np.inf
+    bad = inputs.to_bf16_bits(np.nan_to_num(Xf, nan=0.0, posinf=0.0))
+    bad[7, :] = 0x7FC0            # bf16 quiet NaN
+    bad[130, 3] = 0x7F80          # +inf
+    clean = inputs.to_bf16_bits(np.nan_to_num(Xf, nan=0.0, posinf=0.0))
+    for path in (mr.PATH_TCGEN05, mr.PATH_GENERIC):
+        case.X = bad
+        got = run_gpu(case, path=path)                       # must return; status checked inside run_gpu
+        case.X = clean
+        want = run_gpu(case, path=path)
+        keep = np.ones(300, dtype=bool); keep[[7, 130]] = False
+        assert np.array_equal(got[0][keep], want[0][keep])   # rows without bad values are unaffected
+        assert got[2].sum() <= 300 * 4 and got[2].min() >= 0
