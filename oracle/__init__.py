@@ -44,6 +44,8 @@ def _load():
                                              ctypes.c_int, i32p, f64p]
         lib.more_oracle_logits_at.restype = ctypes.c_int
         lib.more_oracle_threads.restype = ctypes.c_int
+        lib.more_oracle_dispatch.argtypes = [i32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, i64p, i64p]
+        lib.more_oracle_dispatch.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -121,3 +123,17 @@ def logits_at(X, R1, R2, ids) -> np.ndarray:
     if rc != 0:
         raise MemoryError("more_oracle_logits_at failed")
     return out
+
+
+def dispatch(idx, M: int):
+    """Sort + Count of the selected ids ``idx [T][k]``: ``(offsets [M+1], sorted_pairs [number of valid pairs])`` with
+    pairs named by their flat position ``n*k + j``, grouped by expert, ascending within an expert."""
+    lib = _load()
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    T, k = idx.shape
+    offsets = np.zeros((M + 1,), dtype=np.int64)
+    pairs = np.zeros((T * k,), dtype=np.int64)
+    rc = lib.more_oracle_dispatch(_p(idx, ctypes.c_int32), T, k, M, _p(offsets, ctypes.c_int64), _p(pairs, ctypes.c_int64))
+    if rc != 0:
+        raise ValueError("more_oracle_dispatch rejected its arguments")
+    return offsets, pairs[:offsets[M]]

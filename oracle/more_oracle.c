@@ -193,3 +193,29 @@ int more_oracle_route(const uint16_t* X, const uint16_t* R1, const uint16_t* R2,
     }
     return 0;
 }
+
+/*
+ * Dispatch bookkeeping, the "Sort + Count" box of the layer's flowchart (Figure "Operations in the forward pass of
+ * one MoE layer": (N,k) -> (Nk) sorted indices + offsets): the Nk (token, slot) pairs, named by their flat position
+ * p = n*k + j in idx, listed so that their expert ids are non-decreasing, together with where each expert's run
+ * starts.  offsets[e] = number of pairs whose expert id is < e (offsets[M] = number of pairs with a valid id);
+ * sorted_pairs lists, expert by expert, the positions p in ascending order (a stable counting sort).  Pairs whose id
+ * is outside [0, M) are left out.  Plain definition: count, prefix-sum, place.
+ */
+int more_oracle_dispatch(const int32_t* idx, int64_t T, int k, int M, int64_t* offsets, int64_t* sorted_pairs)
+{
+    if (T < 0 || k < 1 || M < 1 || !idx || !offsets || !sorted_pairs) return -1;
+    int64_t* cnt = (int64_t*)calloc((size_t)M + 1, sizeof(int64_t));
+    if (!cnt) return -1;
+    const int64_t n = T * (int64_t)k;
+    for (int64_t p = 0; p < n; ++p)
+        if (idx[p] >= 0 && idx[p] < M) cnt[idx[p]] += 1;
+    int64_t run = 0;
+    for (int e = 0; e < M; ++e) { offsets[e] = run; run += cnt[e]; }
+    offsets[M] = run;
+    for (int e = 0; e < M; ++e) cnt[e] = offsets[e];          /* next free place of each expert's run */
+    for (int64_t p = 0; p < n; ++p)
+        if (idx[p] >= 0 && idx[p] < M) sorted_pairs[cnt[idx[p]]++] = p;
+    free(cnt);
+    return 0;
+}

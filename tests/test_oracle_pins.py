@@ -244,3 +244,25 @@ def test_generator_gives_unit_variance_logits():
     f = np.array([1.0, -2.5, 0.0, 1.00390625, 1.01171875], dtype=np.float32)   # last two: ties at bit 16
     back = inputs.bf16_bits_to_f32(inputs.to_bf16_bits(f))
     assert back.tolist() == [1.0, -2.5, 0.0, 1.0, 1.015625]
+
+
+# --------------------------------------------------------------------------------------------------------
+# Dispatch bookkeeping (Sort + Count): a stable counting sort, pinned against numpy's stable argsort.
+# --------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T,k,M", [(1, 1, 1), (7, 3, 5), (64, 4, 1000), (500, 8, 17)])
+def test_dispatch_matches_stable_argsort(T, k, M):
+    rng = np.random.default_rng(T * 31 + k)
+    idx = rng.integers(0, M, size=(T, k)).astype(np.int32)
+    offsets, pairs = oracle.dispatch(idx, M)
+    flat = idx.ravel()
+    assert np.array_equal(pairs, np.argsort(flat, kind="stable"))
+    assert np.array_equal(offsets, np.concatenate([[0], np.cumsum(np.bincount(flat, minlength=M))]))
+    assert np.all(np.diff(flat[pairs]) >= 0)
+    assert offsets[M] == T * k
+
+
+def test_dispatch_skips_ids_outside_the_expert_range():
+    idx = np.array([[0, 9], [2**31 - 1, 1], [1, -3]], dtype=np.int32)
+    offsets, pairs = oracle.dispatch(idx, 4)
+    assert offsets.tolist() == [0, 1, 3, 3, 3]
+    assert pairs.tolist() == [0, 3, 4]
