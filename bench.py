@@ -358,6 +358,25 @@ def main():
                             plan=vars(mr.more_route_plan(case.T, case.h, case.r, case.M, k))),
                 clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roof)
 
+    # ---- dispatch bookkeeping that follows the router (Sort + Count), same inputs, timed on its own
+    X0, R10, R20, idx0, gate0, counts0 = bufs[0]
+    mr.more_route(X0, R10, R20, k, gate_mode, idx0, gate0, counts0, stream)
+    offs = torch.empty((case.M + 1,), dtype=torch.int32, device="cuda")
+    pairs = torch.empty((case.T * k,), dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(stream)
+    for _ in range(50):
+        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
+    d1.record(stream)
+    stream.synchronize()
+    disp_us = d0.elapsed_time(d1) * 20.0
+    disp_bytes = 8.0 * case.T * k + 12.0 * case.M                # read ids, write pairs; counts in, offsets + cursor out
+    line["dispatch"] = dict(us=disp_us, kernels=["dispatch_scan", "dispatch_scatter"],
+                            algorithmic_gbs=disp_bytes / (disp_us * 1e-6) / 1e9,
+                            hbm_frac=disp_bytes / (disp_us * 1e-6) / 1e9 / peaks["hbm_gbs"])
+
     # ---- context: unfused library-op router on the same inputs
     ms_unfused = None if args.no_context else unfused_reference_ms(torch, bufs, case, gate_mode)
     line["unfused_gpu_reference_ms"] = ms_unfused

@@ -137,6 +137,25 @@ int more_route_noalloc(const void* X, const void* R1, const void* R2,
 long long more_route_noalloc_capacity(void);
 
 /*
+ * more_dispatch -- dispatch bookkeeping for the grouped expert GEMMs that follow the router: the "Sort + Count" box
+ * of the layer's forward flowchart ((N,k) -> (Nk) sorted indices + offsets).
+ *
+ *   idx               device int32 [T][k]: more_route's out_idx.
+ *   counts            device int32 [M]: more_route's out_counts for the same call.
+ *   out_offsets       device int32 [M+1]: out_offsets[e] = number of (token, slot) pairs routed to experts < e, i.e. the
+ *                     exclusive prefix sum of counts; out_offsets[M] = sum of counts (= T*k for finite inputs).
+ *   out_sorted_pairs  device int32 [T*k]: the pairs, named by their flat position p = token*k + slot in idx, grouped by
+ *                     expert: entries out_offsets[e] .. out_offsets[e+1]-1 are exactly the pairs whose id is e.  The
+ *                     order inside one expert's run is unspecified (it depends on the order in which atomic
+ *                     increments land) and may differ from call to call.  Pairs whose id is outside [0, M) (only
+ *                     possible with non-finite inputs) are left out; entries past out_offsets[M] are not written.
+ *   T*k must fit in int32.  Asynchronous on `stream`; uses M*4 bytes of the library's cached scratch, so it must not
+ *   overlap on the GPU with another call of this library on the same device.
+ */
+int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M,
+                  int32_t* out_offsets, int32_t* out_sorted_pairs, void* stream);
+
+/*
  * more_route_plan -- report, without launching, what more_route_ex would do for a shape:
  *   *path_out   MORE_PATH_GENERIC or MORE_PATH_TCGEN05
  *   *msplit_out CTAs per 256-token block (1 on the generic path)

@@ -43,6 +43,8 @@ def lib() -> ctypes.CDLL:
         L.more_route_ex.restype = i32
         L.more_route_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.more_route_host.restype = i32
+        L.more_dispatch.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+        L.more_dispatch.restype = i32
         L.more_route_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.more_route_noalloc.restype = i32
         L.more_route_noalloc_capacity.argtypes = []
@@ -149,6 +151,17 @@ def more_route_noalloc(X, R1, R2, k, gate_mode, out_idx, out_gate, out_counts, s
 
 def more_route_noalloc_capacity() -> int:
     return int(lib().more_route_noalloc_capacity())
+
+
+def more_dispatch(idx, counts, out_offsets, out_sorted_pairs, stream=None):
+    """``more_dispatch`` of the C interface: from ``idx [T,k]`` and ``counts [M]`` (int32, as written by
+    :func:`more_route`) fill ``out_offsets [M+1]`` (exclusive prefix sum of the counts) and ``out_sorted_pairs [T*k]``
+    (flat positions ``token*k + slot`` grouped by expert; order inside an expert's run unspecified)."""
+    T, k = idx.shape
+    M = counts.shape[0]
+    rc = lib().more_dispatch(_ptr(idx), _ptr(counts), T, k, M, _ptr(out_offsets), _ptr(out_sorted_pairs), _stream(stream))
+    if rc != 0:
+        raise MoreRouteError(rc, "more_dispatch")
 
 
 def more_route_status(stream=None) -> int:

@@ -59,6 +59,10 @@ size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p);
 int launch_generic(const RouteArgs& a, DeviceCtx& ctx, void* scratch);
 int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
 
+size_t dispatch_scratch_bytes(int M);
+int launch_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M, int32_t* offsets,
+                    int32_t* sorted_pairs, void* scratch, cudaStream_t stream);
+
 void count_launch(int n = 1);
 
 }  // namespace more

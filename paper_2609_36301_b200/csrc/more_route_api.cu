@@ -216,6 +216,25 @@ int more_route_host(const void* Xh, const void* R1h, const void* R2h, int T, int
     return ok ? MORE_OK : MORE_ERR_CUDA;
 }
 
+int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M, int32_t* out_offsets,
+                  int32_t* out_sorted_pairs, void* stream)
+{
+    if (T < 0 || k < 1 || M < 1 || k > MORE_K_MAX) return MORE_ERR_SHAPE;
+    if ((long long)T * k > 0x7fffffffLL) return MORE_ERR_TOO_LARGE;            // pairs are named by int32 positions
+    if (!counts || !out_offsets) return MORE_ERR_NULL;
+    if (T > 0 && (!idx || !out_sorted_pairs)) return MORE_ERR_NULL;
+    if (!aligned(idx, 4) || !aligned(counts, 4) || !aligned(out_offsets, 4) || !aligned(out_sorted_pairs, 4))
+        return MORE_ERR_ALIGN;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, dispatch_scratch_bytes(M));
+    if (rc != MORE_OK) return rc;
+    return launch_dispatch(idx, counts, T, k, M, out_offsets, out_sorted_pairs, ctx->scratch,
+                           static_cast<cudaStream_t>(stream));
+}
+
 int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int* path_out,
                     int* msplit_out, int* ctas_out)
 {
