@@ -44,6 +44,8 @@ def _load():
                                              ctypes.c_int, i32p, f64p]
         lib.more_oracle_logits_at.restype = ctypes.c_int
         lib.more_oracle_threads.restype = ctypes.c_int
+        lib.more_oracle_psum.argtypes = [u16p, u16p, u16p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, ctypes.c_int, f64p, f64p]
+        lib.more_oracle_psum.restype = ctypes.c_int
         lib.more_oracle_dispatch.argtypes = [i32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, i64p, i64p]
         lib.more_oracle_dispatch.restype = ctypes.c_int
         _lib = lib
@@ -137,3 +139,17 @@ def dispatch(idx, M: int):
     if rc != 0:
         raise ValueError("more_oracle_dispatch rejected its arguments")
     return offsets, pairs[:offsets[M]]
+
+
+def psum(X, R1, R2):
+    """Column sums of the softmax over all experts, ``psum[i] = sum_n P[n, i]`` (Algorithm 2's statistic), and the
+    per-token log-sum-exp: ``(psum [M], lse [T])``."""
+    lib = _load()
+    X, R1, R2, T, h, r, M = _check(X, R1, R2)
+    out = np.zeros((M,), dtype=np.float64)
+    lse = np.zeros((T,), dtype=np.float64)
+    rc = lib.more_oracle_psum(_p(X, ctypes.c_uint16), _p(R1, ctypes.c_uint16), _p(R2, ctypes.c_uint16),
+                              T, h, r, M, _p(out, ctypes.c_double), _p(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError("more_oracle_psum rejected its arguments")
+    return out, lse

@@ -219,3 +219,33 @@ int more_oracle_dispatch(const int32_t* idx, int64_t T, int k, int M, int64_t* o
     free(cnt);
     return 0;
 }
+
+/*
+ * Training-forward statistic of Algorithm 2: the column sums of the row-wise softmax over all M experts,
+ *      psum[i] = sum_n P_{n,i},   P_{n,i} = exp(l_{n,i}) / sum_j exp(l_{n,j})        (Eq. app_softmax, Eq. app_psum),
+ * which is all the Switch balancing loss L_bal = (M/N) f . psum (Eq. app_lbal) needs besides the counts.  Plain
+ * definition: for every token the full logit row, its maximum m and normaliser Z (two passes), then one exp per
+ * entry.  Also returns lse[n] = m + log Z when lse is not NULL.  Serial over tokens (psum is a shared accumulator).
+ */
+int more_oracle_psum(const uint16_t* X, const uint16_t* R1, const uint16_t* R2,
+                     int64_t T, int h, int r, int M, double* psum, double* lse)
+{
+    if (T < 0 || h < 1 || r < 1 || M < 1 || !psum) return -1;
+    double* R1d = widen(R1, (size_t)h * r);
+    double* R2d = widen(R2, (size_t)r * M);
+    double* z = (double*)malloc((size_t)r * sizeof(double));
+    double* l = (double*)malloc((size_t)M * sizeof(double));
+    if (!R1d || !R2d || !z || !l) { free(R1d); free(R2d); free(z); free(l); return -1; }
+    for (int i = 0; i < M; ++i) psum[i] = 0.0;
+    for (int64_t n = 0; n < T; ++n) {
+        token_logits(X + (size_t)n * h, R1d, R2d, h, r, M, z, l);
+        double m = l[0];
+        for (int j = 1; j < M; ++j) if (l[j] > m) m = l[j];
+        double Z = 0.0;
+        for (int j = 0; j < M; ++j) Z += exp(l[j] - m);
+        for (int j = 0; j < M; ++j) psum[j] += exp(l[j] - m) / Z;
+        if (lse) lse[n] = m + log(Z);
+    }
+    free(R1d); free(R2d); free(z); free(l);
+    return 0;
+}

@@ -266,3 +266,37 @@ def test_dispatch_skips_ids_outside_the_expert_range():
     offsets, pairs = oracle.dispatch(idx, 4)
     assert offsets.tolist() == [0, 1, 3, 3, 3]
     assert pairs.tolist() == [0, 3, 4]
+
+
+# --------------------------------------------------------------------------------------------------------
+# Algorithm 2's statistic psum = column sums of the full softmax (Eq. app_psum) and the Switch loss built on it.
+# --------------------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("T,h,r,M", [(1, 8, 2, 3), (50, 32, 8, 130), (256, 128, 8, 256)])
+def test_psum_matches_numpy_softmax_column_sums(T, h, r, M):
+    case = inputs.gaussian_case(T, h, r, M, 1, 1, seed=21)
+    ps, lse = oracle.psum(case.X, case.R1, case.R2)
+    L = (inputs.bf16_bits_to_f64(case.X) @ inputs.bf16_bits_to_f64(case.R1)) @ inputs.bf16_bits_to_f64(case.R2)
+    np.testing.assert_allclose(ps, softmax(L, axis=1).sum(axis=0), rtol=1e-12)
+    np.testing.assert_allclose(lse, logsumexp(L, axis=1), rtol=0, atol=1e-12)
+    np.testing.assert_allclose(ps.sum(), T, rtol=1e-12)                    # every row of P sums to one
+    assert np.array_equal(lse, oracle.route(case.X, case.R1, case.R2, 1, 1).lse)   # same row statistics as the router
+
+
+def test_psum_uniform_router_gives_unit_switch_loss():
+    # all-zero expert vectors: P = 1/M everywhere, psum = T/M, and L_bal = (M/N) f . psum = 1 for any dispatch f
+    case = inputs.gaussian_case(40, 16, 4, 12, 3, 1, seed=22)
+    R2 = np.zeros_like(case.R2)
+    ps, _ = oracle.psum(case.X, case.R1, R2)
+    np.testing.assert_allclose(ps, 40 / 12, rtol=1e-14)
+    res = oracle.route(case.X, case.R1, R2, 3, 1)
+    f = res.counts / (40 * 3)
+    np.testing.assert_allclose(12 / 40 * (f @ ps), 1.0, rtol=1e-13)
+    assert np.array_equal(res.idx, np.broadcast_to(np.arange(3), (40, 3)))  # exact ties everywhere: lowest ids
+
+
+def test_psum_is_equivariant_under_expert_relabelling():
+    case = inputs.gaussian_case(30, 24, 6, 41, 2, 1, seed=23)
+    perm = np.random.default_rng(3).permutation(41)
+    a, _ = oracle.psum(case.X, case.R1, case.R2)
+    b, _ = oracle.psum(case.X, case.R1, case.R2[:, perm])
+    np.testing.assert_allclose(b, a[perm], rtol=1e-13)
