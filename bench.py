@@ -377,6 +377,22 @@ def main():
                             algorithmic_gbs=disp_bytes / (disp_us * 1e-6) / 1e9,
                             hbm_frac=disp_bytes / (disp_us * 1e-6) / 1e9 / peaks["hbm_gbs"])
 
+    # ---- Algorithm 2's second sweep (psum = column sums of the full softmax), same inputs, timed on its own
+    lse0 = torch.empty((case.T,), dtype=torch.float32, device="cuda")
+    mr.more_route_ex(X0, R10, R20, k, 1, idx0, gate0, counts0, None, lse0, 0, 0, stream)
+    psum0 = torch.empty((case.M,), dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
+    d0.record(stream)
+    for _ in range(20):
+        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
+    d1.record(stream)
+    stream.synchronize()
+    ps_secs = d0.elapsed_time(d1) * 1e-3 / 20
+    rp = roofline(case.T, case.h, case.r, case.M, k, ps_secs, peaks)
+    line["train_stats_psum"] = dict(us=ps_secs * 1e6, kernel="psum_tcgen05_kernel", bound=rp["bound"],
+                                    roofline_frac=rp["frac"], psum_total=float(psum0.sum()), tokens=case.T)
+
     # ---- context: unfused library-op router on the same inputs
     ms_unfused = None if args.no_context else unfused_reference_ms(torch, bufs, case, gate_mode)
     line["unfused_gpu_reference_ms"] = ms_unfused

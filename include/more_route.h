@@ -137,6 +137,23 @@ int more_route_noalloc(const void* X, const void* R1, const void* R2,
 long long more_route_noalloc_capacity(void);
 
 /*
+ * more_route_psum -- the training-forward statistic of Algorithm 2: psum[i] = sum_n P_{n,i}, the column sums of the
+ * row-wise softmax over all M experts (Eq. app_softmax, Eq. app_psum), from which the Switch balancing loss is
+ * L_bal = (M/N) f . psum with f = counts / (N k) (Eq. app_lbal).  This is Algorithm 2's second sweep: the logit tiles
+ * are produced again (z is recomputed from X, the second contraction runs transposed so that a tensor-memory lane is
+ * an expert) and reduced over the tokens on chip; nothing of size T x M is written.
+ *
+ *   X, R1, R2, T, h, r, M   as for more_route (device, bf16).
+ *   lse        device fp32 [T]: every token's log-sum-exp over all M logits, as written to out_lse by more_route_ex
+ *              for the same inputs (P_{n,i} = exp(l_{n,i} - lse_n)).
+ *   out_psum   device fp32 [M]: OVERWRITTEN (zeroed on `stream`, then accumulated with floating-point atomics, so the
+ *              last bits depend on the order in which the adds land; the sum over all experts is T up to rounding).
+ *   path       MORE_PATH_*, as for more_route_ex (the tensor-core path needs h, r, M multiples of 8 and r <= 64).
+ */
+int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h, int r, int M,
+                    const float* lse, float* out_psum, int path, void* stream);
+
+/*
  * more_dispatch -- dispatch bookkeeping for the grouped expert GEMMs that follow the router: the "Sort + Count" box
  * of the layer's forward flowchart ((N,k) -> (Nk) sorted indices + offsets).
  *

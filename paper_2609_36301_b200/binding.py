@@ -43,6 +43,8 @@ def lib() -> ctypes.CDLL:
         L.more_route_ex.restype = i32
         L.more_route_host.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.more_route_host.restype = i32
+        L.more_route_psum.argtypes = [vp, vp, vp, i32, i32, i32, i32, vp, vp, i32, vp]
+        L.more_route_psum.restype = i32
         L.more_dispatch.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.more_dispatch.restype = i32
         L.more_route_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -151,6 +153,16 @@ def more_route_noalloc(X, R1, R2, k, gate_mode, out_idx, out_gate, out_counts, s
 
 def more_route_noalloc_capacity() -> int:
     return int(lib().more_route_noalloc_capacity())
+
+
+def more_route_psum(X, R1, R2, lse, out_psum, path=PATH_AUTO, stream=None):
+    """``more_route_psum`` of the C interface: ``out_psum [M]`` (fp32, overwritten) = column sums of the softmax over
+    all experts, given every token's ``lse [T]`` from :func:`more_route_ex` on the same inputs (Algorithm 2)."""
+    T, h = X.shape
+    r, M = R2.shape
+    rc = lib().more_route_psum(_ptr(X), _ptr(R1), _ptr(R2), T, h, r, M, _ptr(lse), _ptr(out_psum), path, _stream(stream))
+    if rc != 0:
+        raise MoreRouteError(rc, "more_route_psum")
 
 
 def more_dispatch(idx, counts, out_offsets, out_sorted_pairs, stream=None):

@@ -59,6 +59,11 @@ size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p);
 int launch_generic(const RouteArgs& a, DeviceCtx& ctx, void* scratch);
 int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
 
+int launch_generic_psum(const __nv_bfloat16* X, const __nv_bfloat16* R1, const __nv_bfloat16* R2, int T, int h, int r,
+                        int M, const float* lse, float* psum, void* scratch, cudaStream_t stream);
+int launch_psum_tcgen05(const __nv_bfloat16* X, const __nv_bfloat16* R1, const __nv_bfloat16* R2, int T, int h, int r,
+                        int M, const float* lse, float* psum, DeviceCtx& ctx, cudaStream_t stream);
+
 size_t dispatch_scratch_bytes(int M);
 int launch_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M, int32_t* offsets,
                     int32_t* sorted_pairs, void* scratch, cudaStream_t stream);

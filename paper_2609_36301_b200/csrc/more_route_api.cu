@@ -216,6 +216,36 @@ int more_route_host(const void* Xh, const void* R1h, const void* R2h, int T, int
     return ok ? MORE_OK : MORE_ERR_CUDA;
 }
 
+int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h, int r, int M, const float* lse,
+                    float* out_psum, int path, void* stream)
+{
+    if (path != MORE_PATH_AUTO && path != MORE_PATH_GENERIC && path != MORE_PATH_TCGEN05) return MORE_ERR_MODE;
+    if (T < 0 || h < 1 || r < 1 || M < 1 || r > MORE_R_MAX) return MORE_ERR_SHAPE;
+    if (!out_psum) return MORE_ERR_NULL;
+    if (T > 0 && (!X || !R1 || !R2 || !lse)) return MORE_ERR_NULL;
+    if (!aligned(X, 16) || !aligned(R1, 16) || !aligned(R2, 16) || !aligned(lse, 4) || !aligned(out_psum, 4))
+        return MORE_ERR_ALIGN;
+    const bool fast_ok = tcgen05_shape_ok(T, h, r, M, 1);
+    if (path == MORE_PATH_TCGEN05 && !fast_ok) return MORE_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool fast = fast_ok && path != MORE_PATH_GENERIC;
+    if (!fast) {
+        rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, (size_t)T * r * sizeof(float));
+        if (rc != MORE_OK) return rc;
+    }
+    if (cudaMemsetAsync(out_psum, 0, (size_t)M * sizeof(float), st) != cudaSuccess) return MORE_ERR_CUDA;
+    if (T == 0) return MORE_OK;
+    const __nv_bfloat16* x = static_cast<const __nv_bfloat16*>(X);
+    const __nv_bfloat16* r1 = static_cast<const __nv_bfloat16*>(R1);
+    const __nv_bfloat16* r2 = static_cast<const __nv_bfloat16*>(R2);
+    return fast ? launch_psum_tcgen05(x, r1, r2, T, h, r, M, lse, out_psum, *ctx, st)
+                : launch_generic_psum(x, r1, r2, T, h, r, M, lse, out_psum, ctx->scratch, st);
+}
+
 int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M, int32_t* out_offsets,
                   int32_t* out_sorted_pairs, void* stream)
 {

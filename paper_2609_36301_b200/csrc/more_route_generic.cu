@@ -101,7 +101,35 @@ __global__ void generic_route_tokens(const float* __restrict__ Z, const __nv_bfl
     if (out_lse && lane == 0) out_lse[n] = m_all + logf(z_all);
 }
 
+// psum[j] += sum over a chunk of tokens of exp(l_{n,j} - lse_n): thread per expert, 256 tokens per block row.
+__global__ void generic_psum_kernel(const float* __restrict__ Z, const __nv_bfloat16* __restrict__ R2,
+                                    const float* __restrict__ lse, int T, int r, int M, float* __restrict__ psum)
+{
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    const int n0 = blockIdx.y * 256, n1 = min(T, n0 + 256);
+    if (j >= M) return;
+    float acc = 0.f;
+    for (int n = n0; n < n1; ++n) {
+        const float* z = Z + (int64_t)n * r;
+        float l = 0.f;
+        for (int i = 0; i < r; ++i) l = fmaf(z[i], __bfloat162float(R2[(int64_t)i * M + j]), l);
+        acc += expf(l - lse[n]);
+    }
+    atomicAdd(psum + j, acc);
+}
+
 }  // namespace
+
+int launch_generic_psum(const __nv_bfloat16* X, const __nv_bfloat16* R1, const __nv_bfloat16* R2, int T, int h, int r,
+                        int M, const float* lse, float* psum, void* scratch, cudaStream_t stream)
+{
+    float* Z = static_cast<float*>(scratch);
+    generic_project_z<<<T, 128, 0, stream>>>(X, R1, Z, h, r);
+    dim3 grid((M + 127) / 128, (T + 255) / 256);
+    generic_psum_kernel<<<grid, 128, 0, stream>>>(Z, R2, lse, T, r, M, psum);
+    count_launch(2);
+    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
 
 size_t generic_scratch_bytes(const RouteArgs& a) { return (size_t)a.T * (size_t)a.r * sizeof(float); }
 
