@@ -175,7 +175,7 @@ struct KernelParams {
 // Final outputs of one token from its sorted list and (m2, z): m2 is the running max in log2 units.
 template <int KCAP>
 __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, const TopList<KCAP>& L, float m2,
-                                            float zsum)
+                                            float zsum, int* hist)
 {
     constexpr float kLn2 = 0.6931471805599453f, kLog2e = 1.4426950408889634f;
     const int k = p.k;
@@ -195,7 +195,8 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
             p.out_idx[row * k + q] = L.id[q];
             p.out_gate[row * k + q] = ex2f(L.v[q] * kLog2e - ref2) * inv;
             if (p.out_topval) p.out_topval[row * k + q] = L.v[q];
-            if ((unsigned)L.id[q] < (unsigned)p.M) atomicAdd(p.out_counts + L.id[q], 1);   // (non-finite inputs can leave a slot unfilled)
+            if ((unsigned)L.id[q] < (unsigned)p.M)            // (non-finite inputs can leave a slot unfilled)
+                atomicAdd((hist ? hist : p.out_counts) + L.id[q], 1);
         }
     }
     if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
@@ -519,9 +520,32 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
         // ---- finish.  All 256 epilogue threads meet here, also after an abort, so the decision is uniform.
         asm volatile("bar.sync 1, 256;" ::: "memory");
+        // Expert histogram: when the M bins fit into the (now idle) ring, the CTA counts its tokens' ids in shared
+        // memory and flushes only the non-zero bins with one global atomic each; otherwise straight to global memory
+        // (with that many experts the bins hardly collide).  With few experts thousands of pairs hit each bin, and
+        // same-address global atomics would serialise.
+        int* hist = (p.M * 4 <= kRingBytes) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
+        const int etid = threadIdx.x - 64;                   // 0..255 among the epilogue threads
+        auto hist_clear = [&]() {
+            if (hist) {
+                for (int e = etid; e < p.M; e += kEpilogueThreads) hist[e] = 0;
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+            }
+        };
+        auto hist_flush = [&]() {
+            if (hist) {
+                asm volatile("bar.sync 1, 256;" ::: "memory");
+                for (int e = etid; e < p.M; e += kEpilogueThreads) {
+                    const int c = hist[e];
+                    if (c) atomicAdd(p.out_counts + e, c);
+                }
+            }
+        };
         if (*abort_flag == 0) {
             if (p.msplit == 1) {
-                if (row_live) write_token<KCAP>(p, row, L, m2, zsum);
+                hist_clear();
+                if (row_live) write_token<KCAP>(p, row, L, m2, zsum, hist);
+                hist_flush();
             } else {
                 // park the partial list; the CTA that arrives last for this token block merges all of them
                 const int64_t slot = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit + split;
@@ -557,7 +581,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                             gm = nm;
                         }
                     }
-                    if (row_live) write_token<KCAP>(p, row, G, gm, gz);
+                    hist_clear();
+                    if (row_live) write_token<KCAP>(p, row, G, gm, gz, hist);
+                    hist_flush();
                     if (threadIdx.x == 64) p.counters[blk] = 0;   // ready for the next call
                 }
             }
