@@ -246,6 +246,45 @@ def unfused_reference_ms(torch, bufs, case, gate_mode, iters=5):
         return None
 
 
+def extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line):
+    """Times the library's other entry points on the same inputs, each on its own (outside the router's timed region):
+    the dispatch bookkeeping that follows the router (Sort + Count) and Algorithm 2's second sweep (psum)."""
+    X0, R10, R20, idx0, gate0, counts0 = bufs[0]
+    mr.more_route(X0, R10, R20, k, gate_mode, idx0, gate0, counts0, stream)
+    offs = torch.empty((case.M + 1,), dtype=torch.int32, device="cuda")
+    pairs = torch.empty((case.T * k,), dtype=torch.int32, device="cuda")
+    for _ in range(3):
+        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    d0.record(stream)
+    for _ in range(50):
+        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
+    d1.record(stream)
+    stream.synchronize()
+    disp_us = d0.elapsed_time(d1) * 20.0
+    disp_bytes = 8.0 * case.T * k + 12.0 * case.M                # read ids, write pairs; counts in, offsets + cursor out
+    line["dispatch"] = dict(us=disp_us, kernels=["dispatch_scan", "dispatch_scatter"],
+                            algorithmic_gbs=disp_bytes / (disp_us * 1e-6) / 1e9,
+                            hbm_frac=disp_bytes / (disp_us * 1e-6) / 1e9 / peaks["hbm_gbs"])
+
+    # ---- Algorithm 2's second sweep (psum = column sums of the full softmax), same inputs, timed on its own
+    lse0 = torch.empty((case.T,), dtype=torch.float32, device="cuda")
+    mr.more_route_ex(X0, R10, R20, k, 1, idx0, gate0, counts0, None, lse0, 0, 0, stream)
+    psum0 = torch.empty((case.M,), dtype=torch.float32, device="cuda")
+    for _ in range(3):
+        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
+    d0.record(stream)
+    for _ in range(20):
+        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
+    d1.record(stream)
+    stream.synchronize()
+    ps_secs = d0.elapsed_time(d1) * 1e-3 / 20
+    rp = roofline(case.T, case.h, case.r, case.M, k, ps_secs, peaks)
+    line["train_stats_psum"] = dict(us=ps_secs * 1e6, kernel="psum_tcgen05_kernel", bound=rp["bound"],
+                                    roofline_frac=rp["frac"], psum_total=float(psum0.sum()), tokens=case.T)
+
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -256,7 +295,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-others", action="store_true", help="skip the per-configuration table")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-context", action="store_true", help="skip the unfused library-op router (context only)")
+    ap.add_argument("--no-context", action="store_true",
+                    help="router only: skip the dispatch / psum entry points and the unfused library-op router")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
 
@@ -358,40 +398,8 @@ def main():
                             plan=vars(mr.more_route_plan(case.T, case.h, case.r, case.M, k))),
                 clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roof)
 
-    # ---- dispatch bookkeeping that follows the router (Sort + Count), same inputs, timed on its own
-    X0, R10, R20, idx0, gate0, counts0 = bufs[0]
-    mr.more_route(X0, R10, R20, k, gate_mode, idx0, gate0, counts0, stream)
-    offs = torch.empty((case.M + 1,), dtype=torch.int32, device="cuda")
-    pairs = torch.empty((case.T * k,), dtype=torch.int32, device="cuda")
-    for _ in range(3):
-        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
-    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    d0.record(stream)
-    for _ in range(50):
-        mr.more_dispatch(idx0, counts0, offs, pairs, stream)
-    d1.record(stream)
-    stream.synchronize()
-    disp_us = d0.elapsed_time(d1) * 20.0
-    disp_bytes = 8.0 * case.T * k + 12.0 * case.M                # read ids, write pairs; counts in, offsets + cursor out
-    line["dispatch"] = dict(us=disp_us, kernels=["dispatch_scan", "dispatch_scatter"],
-                            algorithmic_gbs=disp_bytes / (disp_us * 1e-6) / 1e9,
-                            hbm_frac=disp_bytes / (disp_us * 1e-6) / 1e9 / peaks["hbm_gbs"])
-
-    # ---- Algorithm 2's second sweep (psum = column sums of the full softmax), same inputs, timed on its own
-    lse0 = torch.empty((case.T,), dtype=torch.float32, device="cuda")
-    mr.more_route_ex(X0, R10, R20, k, 1, idx0, gate0, counts0, None, lse0, 0, 0, stream)
-    psum0 = torch.empty((case.M,), dtype=torch.float32, device="cuda")
-    for _ in range(3):
-        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
-    d0.record(stream)
-    for _ in range(20):
-        mr.more_route_psum(X0, R10, R20, lse0, psum0, 0, stream)
-    d1.record(stream)
-    stream.synchronize()
-    ps_secs = d0.elapsed_time(d1) * 1e-3 / 20
-    rp = roofline(case.T, case.h, case.r, case.M, k, ps_secs, peaks)
-    line["train_stats_psum"] = dict(us=ps_secs * 1e6, kernel="psum_tcgen05_kernel", bound=rp["bound"],
-                                    roofline_frac=rp["frac"], psum_total=float(psum0.sum()), tokens=case.T)
+    if not args.no_context:
+        extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line)
 
     # ---- context: unfused library-op router on the same inputs
     ms_unfused = None if args.no_context else unfused_reference_ms(torch, bufs, case, gate_mode)
