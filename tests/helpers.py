@@ -1,6 +1,7 @@
 """Shared checking code of the GPU parity tests: the acceptance rule, written once.
 
-Acceptance rule (tolerances are the benchmark definition's, the reasoning is in the design doc):
+Acceptance rule (the 1e-3 near-tie exemption and the 2e-3 gate tolerance are the benchmark definition's; the GPU's
+logits are good to ~4e-5 because z is carried as a bf16 high part plus a bf16 low part and accumulated in fp32):
   * a token is *exempt* when the oracle's k-th and (k+1)-th logits differ by less than 1e-3;
   * non-exempt tokens: the GPU's set of expert ids equals the oracle's exactly;
   * exempt tokens: ids distinct and in range, every chosen expert's oracle logit >= l_(k) - 1e-3, and every
