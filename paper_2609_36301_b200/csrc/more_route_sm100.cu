@@ -7,22 +7,25 @@
 //
 //   phase 1  z = X_blk R1            TMA streams 256x64 X tiles and 64x64 R1 tiles (zero-filled beyond r),
 //                                    tcgen05.mma accumulates two 128 x 64 fp32 blocks in TMEM.
-//   narrow   z -> bf16 hi + bf16 lo  written to shared memory as the K-major A operands [hi | lo].  Carrying both
-//                                    parts keeps the logits within ~3e-5 of exact arithmetic.
-//   phase 2  y = z R2[:, tile]       one 128-expert tile at a time: TMA brings the r x 128 slice of R2 once for
-//                                    both accumulators (this halves the L2 traffic of re-reading R2 per token
-//                                    block), tcgen05.mma (hi then lo into the same accumulator) fills TMEM,
-//                                    the epilogue drains it: TMEM lane = token, so each epilogue thread owns one
-//                                    token and reads its logits 32 columns at a time.
-//   merge    running top-k           sorted (value, id) list in registers, fed through a small per-token candidate
-//                                    buffer in shared memory (see Selector).
+//   narrow   z -> bf16 hi + bf16 lo  written back to tensor memory (tcgen05.st) as the A operands [hi | lo] of phase 2:
+//                                    TMEM lane = token, two K-elements per 32-bit column.  Carrying both parts keeps
+//                                    the logits within ~3e-5 of exact arithmetic.
+//   phase 2  y = z R2[:, block]      64 experts at a time: TMA brings the r x 64 block of R2 once for both
+//                                    accumulators, tcgen05.mma with A from tensor memory (hi then lo into the same
+//                                    accumulator) fills 64 TMEM columns, the epilogue drains them: each epilogue
+//                                    thread owns one token and reads its logits 16 columns at a time.  The group hands
+//                                    the accumulator back as soon as the last 32 columns are in registers, so the next
+//                                    step's MMAs run while those are processed.
+//   merge    running top-k           sorted (value, id) list in registers, fed through a per-token candidate buffer
+//                                    in shared memory (see Selector).
 //   finish   gates, ids, counts      written by the CTA itself (msplit == 1) or, after the partial lists have been
 //                                    parked in scratch, by whichever CTA of the token block finishes last.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue, warps 2..9 = epilogue (warp w reads
-// TMEM lanes 32*(w%4).. of accumulator (w-2)/4).  Two CTAs are resident per SM (256 TMEM columns and ~112 KB of
-// shared memory each): while one CTA's epilogue drains its accumulators the other CTA's MMAs run, and one CTA's
-// HBM-bound phase 1 overlaps the other's expert sweep.
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue (the whole warp stays converged and one
+// elected lane issues; see tc_mma_bf16_ts_elect), warps 2..9 = epilogue (warp w reads TMEM lanes 32*(w%4).. of
+// accumulator (w-2)/4).  Two CTAs are resident per SM (256 TMEM columns and ~112 KB of shared memory each): while one
+// group's epilogue drains its accumulator the MMAs of the other three groups of the SM run, and one CTA's HBM-bound
+// phase 1 overlaps the other's expert sweep.
 //
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
 // status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
@@ -76,15 +79,21 @@ struct TopList {
     }
 };
 
-// Running top-k of one token.  Between refreshes the sorted list is left alone: elements that beat the cached
-// threshold `tau` (the list's last entry as of the last refresh) are only appended, in ascending column order, to
-// this thread's column of a shared-memory candidate buffer (one predicated 8-byte store each); refresh() then
-// inserts them one by one, so the inserts of several chunks of all 32 tokens of a warp are executed together.
-constexpr int kCandSlotStride = kEpilogueThreads * 8;     // bytes between successive slots of one thread
-#ifndef MORE_WARN
-#define MORE_WARN 2
+// Running top-k of one token.  Between refreshes the sorted list is left alone.  A chunk of 16 logits is looked at
+// as five triples and a single; every group whose maximum beats the cached threshold `tau` (the list's last entry
+// as of the last refresh, hence never above the true threshold) is appended whole, in ascending column order, to
+// this thread's column of a shared-memory candidate buffer: one predicated 16-byte store {v0, v1, v2, first column}
+// and no branch.  refresh() then inserts the buffered elements that beat the up-to-date threshold, so the inserts of
+// several chunks of all 32 tokens of a warp are executed together.  A chunk appends at most 6 entries and the warp
+// refreshes as soon as some token has fewer than 6 free slots left, so the buffer cannot overflow.
+constexpr int kCandSlotStride = kEpilogueThreads * 16;    // bytes between successive slots of one thread
+#ifndef MORE_CAND_CAP
+#define MORE_CAND_CAP 14
 #endif
-constexpr int kRefreshAt = MORE_WARN;                     // a warp folds its buffers once some token holds this many
+#ifndef MORE_WARN
+#define MORE_WARN (MORE_CAND_CAP - 6)
+#endif
+static_assert(MORE_WARN >= 1 && MORE_WARN <= MORE_CAND_CAP - 6, "a chunk must always find 6 free slots");
 constexpr unsigned kFullMask = 0xffffffffu;
 
 template <int KCAP, int CAP>
@@ -93,7 +102,6 @@ struct Selector {
     float tau;
     uint32_t ptr;     // shared-memory address of this thread's next free candidate slot
     uint32_t base;    // its first slot
-    uint32_t lim;     // ptr is clamped here after every triple; reaching it means "may have lost candidates"
     uint32_t warn;    // at or beyond this fill level the warp refreshes after the chunk
 
     __device__ __forceinline__ void init(uint32_t first_slot)
@@ -101,56 +109,48 @@ struct Selector {
         L.init();
         tau = -INFINITY;
         base = ptr = first_slot;
-        lim = first_slot + (CAP - 3) * kCandSlotStride;
-        warn = first_slot + (kRefreshAt < CAP - 3 ? kRefreshAt : CAP - 3) * kCandSlotStride;
+        warn = first_slot + MORE_WARN * kCandSlotStride;
     }
     __device__ __forceinline__ void refresh()
     {
         for (uint32_t a = base; a < ptr; a += kCandSlotStride) {
-            float x;
-            int j;
-            asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=f"(x), "=r"(j) : "r"(a) : "memory");
-            L.insert(x, j);
+            float x0, x1, x2;
+            int col;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=r"(col) : "r"(a) : "memory");
+            const float m = max3(x0, x1, x2);
+            if (m > L.tau()) {
+                // the group's maximum first (its lowest column on a tie), then, rarely, the other two in column order
+                const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : 2);
+                L.insert(m, col + j);
+                const float y0 = (j == 0) ? x1 : x0, y1 = (j == 2) ? x1 : x2;
+                const int c0 = col + ((j == 0) ? 1 : 0), c1 = col + ((j == 2) ? 1 : 2);
+                if (fmaxf(y0, y1) > L.tau()) {
+                    if (y0 > L.tau()) L.insert(y0, c0);
+                    if (y1 > L.tau()) L.insert(y1, c1);
+                }
+            }
         }
         ptr = base;
         tau = L.tau();
     }
-    // if (x > tau) append (x, col)
-    __device__ __forceinline__ void append_if_above(float x, int col)
+    // if (t > tau) append {v0, v1, v2, col}
+    __device__ __forceinline__ void append3(float t, float v0, float v1, float v2, int col)
     {
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "setp.gt.f32 p, %1, %3;\n\t"
-            "@p st.shared.v2.b32 [%0], {%1, %2};\n\t"
-            "@p add.u32 %0, %0, %4;\n\t}"
+            "setp.gt.f32 p, %1, %6;\n\t"
+            "@p st.shared.v4.b32 [%0], {%2, %3, %4, %5};\n\t"
+            "@p add.u32 %0, %0, %7;\n\t}"
             : "+r"(ptr)
-            : "f"(x), "r"(col), "f"(tau), "n"(kCandSlotStride)
+            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "r"(col), "f"(tau), "n"(kCandSlotStride)
             : "memory");
     }
-    // v: 16 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]) for i < 5; v[15] stands
-    // alone.  Appends every element above tau; if the buffer cannot take them all, ptr ends at lim (the caller then
-    // redoes the chunk).
+    // v: 16 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]) for i < 5; v[15] stands alone.
     __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[5], int col0)
     {
-#ifdef MORE_FLAT_SCAN
-        (void)t;
 #pragma unroll
-        for (int i = 0; i < 16; ++i) {
-            append_if_above(v[i], col0 + i);
-            if (i % 3 == 2 || i == 15) ptr = min(ptr, lim);
-        }
-#else
-#pragma unroll
-        for (int i = 0; i < 5; ++i) {
-            if (t[i] > tau) {
-#pragma unroll
-                for (int e = 0; e < 3; ++e) append_if_above(v[3 * i + e], col0 + 3 * i + e);
-                ptr = min(ptr, lim);
-            }
-        }
-        append_if_above(v[15], col0 + 15);
-        ptr = min(ptr, lim);
-#endif
+        for (int i = 0; i < 5; ++i) append3(t[i], v[3 * i], v[3 * i + 1], v[3 * i + 2], col0 + 3 * i);
+        append3(v[15], v[15], -INFINITY, -INFINITY, col0 + 15);
     }
 };
 
@@ -209,13 +209,15 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                      const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
 {
     constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
-    constexpr int kZopOne = (RPAD == 64) ? 32768 : 16384;       // A operand [hi | lo] of one 128-token accumulator
-    constexpr int kZopBytes = 2 * kZopOne;
-    constexpr int kR2StageBytes = RPAD * 256;                   // one 128-expert tile: two 64-expert blocks of RPAD rows x 128 B
-    constexpr int kStagesP2 = (RPAD == 64) ? 2 : 4;             // tiles in flight
-    constexpr int kCandCap = (RPAD == 64) ? 7 : 16;             // candidate slots per token (what the ring has room for)
+    constexpr int kHalf = 64;                                   // experts per phase-2 step: one 128-byte-wide R2 block
+    constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
+    constexpr int kStagesP2 = (RPAD == 64) ? 6 : 8;             // R2 blocks in flight
+    constexpr int kCandCap = MORE_CAND_CAP;                     // candidate slots per token
     constexpr int kCandBytes = kCandCap * kCandSlotStride;
-    static_assert(kZopBytes + kCandBytes + kStagesP2 * kR2StageBytes <= kRingBytes, "phase-2 layout does not fit");
+    static_assert(kCandBytes + kStagesP2 * kR2StageBytes <= kRingBytes, "phase-2 layout does not fit");
+    // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
+    // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.
+    constexpr uint32_t kAccCols = 64, kZopCol0 = 128;
     constexpr float kLog2e = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
@@ -240,7 +242,6 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // expert tiles of this CTA: an even share of ceil(M/128) tiles
     const int tile_lo = (int)(((long long)p.tiles_total * split) / p.msplit);
     const int tile_hi = (int)(((long long)p.tiles_total * (split + 1)) / p.msplit);
-    const int ntiles = tile_hi - tile_lo;
     const int ktiles1 = (p.h + 63) / 64;
 
     if (threadIdx.x == 0) {
@@ -263,9 +264,12 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t zop = ring;                                  // phase 2: A operands, accumulator 0 then 1
-    const uint32_t cand = ring + kZopBytes;                     // phase 2: candidate buffers
-    const uint32_t r2ring = ring + kZopBytes + kCandBytes;      // phase 2: R2 stages
+    const uint32_t cand = ring;                                 // phase 2: candidate buffers
+    const uint32_t r2ring = ring + kCandBytes;                  // phase 2: R2 stages
+    // 64-expert steps of this CTA (the last one of the last tile is skipped when it lies wholly beyond M)
+    const int e_lo = tile_lo * kTileExperts;
+    const int e_hi = min(tile_hi * kTileExperts, p.M);
+    const int nsteps = (e_hi - e_lo + kHalf - 1) / kHalf;
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
@@ -282,67 +286,64 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             }
             // the ring is reused by phase 2: wait until every phase-1 MMA has finished reading it
             ok = ok && mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
-            for (int it = 0; it < ntiles && ok; ++it) {
+            for (int it = 0; it < nsteps && ok; ++it) {
                 const int s = it % kStagesP2;
                 if (it >= kStagesP2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it / kStagesP2) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t dst = r2ring + s * kR2StageBytes;
-                const int e0 = (tile_lo + it) * kTileExperts;
                 mbar_expect_tx(bar(B_FULL2 + s), kR2StageBytes);
-                tma_load_2d(dst, &map_r2, bar(B_FULL2 + s), e0, 0);
-                tma_load_2d(dst + RPAD * 128, &map_r2, bar(B_FULL2 + s), e0 + 64, 0);
+                tma_load_2d(r2ring + s * kR2StageBytes, &map_r2, bar(B_FULL2 + s), e_lo + it * kHalf, 0);
             }
         }
     } else if (warp == 1) {
         // ======================================================================================= MMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            constexpr uint32_t idesc1 = umma_idesc(64);
-            constexpr uint32_t idesc2 = umma_idesc(kTileExperts);
+        // The whole warp runs this code converged; one elected lane issues each tcgen05 instruction.
+        bool ok = true;
+        constexpr uint32_t idesc1 = umma_idesc(64);
+        constexpr uint32_t idesc2 = umma_idesc(kHalf);
+        {
+            // descriptor words of stage 0: K-major X tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address
+            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
+            const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
                 const int s = kt % kStagesP1;
-                ok = mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status);
+                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t xa = ring + s * kP1StageBytes, rb = xa + kXTileBytes;
+                const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), r_lo = r_lo0 + s * (kP1StageBytes >> 4);
 #pragma unroll
                 for (int a = 0; a < 2; ++a) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t ad = umma_desc_sw128(xa + a * 16384 + kk * 32, 16, 1024);   // K-major, +32 B per K=16
-                        const uint64_t bd = umma_desc_sw128(rb + kk * 2048, 8192, 1024);           // MN-major, 16 K-rows
-                        tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc1, (kt | kk) != 0);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
+                        tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
+                                             r_lo + kk * (2048 >> 4), r_hi, idesc1, (kt | kk) != 0);
                 }
-                tc_commit(bar(B_EMPTY1 + s));
+                tc_commit_elect(bar(B_EMPTY1 + s));
             }
-            if (ok) tc_commit(bar(B_ZACC));
-            ok = ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status);
-            tc_fence_after();
-            for (int it = 0; it < ntiles && ok; ++it) {
-                const int s = it % kStagesP2;
-                ok = mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status);
-                if (!ok) break;
-                const uint32_t rb = r2ring + s * kR2StageBytes;
+        }
+        if (ok) tc_commit_elect(bar(B_ZACC));
+        ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status));
+        tc_fence_after();
+        const uint64_t bd0 = umma_desc_sw128(r2ring, 8192, 1024);
+        const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+        for (int it = 0; it < nsteps && ok; ++it) {
+            const int s = it % kStagesP2;
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status));
+            if (!ok) break;
+            const uint32_t b_lo = b_lo0 + s * (kR2StageBytes >> 4);
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {
-                    // accumulator a is free once its 128 epilogue threads have drained the previous tile
-                    ok = ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int j = 0; j < 2 * kKSteps; ++j) {
-                        const uint32_t abyte = j * 32;                                       // K offset in [hi | lo]
-                        const uint64_t ad =
-                            umma_desc_sw128(zop + a * kZopOne + (abyte >> 7) * 16384 + (abyte & 127), 16, 1024);
-                        const uint64_t bd = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
-                        tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc2, j != 0);
-                    }
-                    tc_commit(bar(B_ACCF + a));
-                }
+            for (int a = 0; a < 2; ++a) {
+                // accumulator a is free once its 128 epilogue threads have read the previous step out of it
+                ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
                 if (!ok) break;
-                tc_commit(bar(B_EMPTY2 + s));
+                tc_fence_after();
+#pragma unroll
+                for (int j = 0; j < 2 * kKSteps; ++j)       // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
+                    tc_mma_bf16_ts_elect(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64 + j * 8,
+                                         b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
+                tc_commit_elect(bar(B_ACCF + a));
             }
+            if (!ok) break;
+            tc_commit_elect(bar(B_EMPTY2 + s));
         }
     } else {
         // ========================================================================================= epilogue
@@ -353,12 +354,12 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int64_t row = (int64_t)tok0 + row_in_blk;
         const bool row_live = row_in_blk < p.block_tokens && row < p.T;     // rows past the block belong to the next CTA
         const bool warp_live = acc * 128 + q * 32 < p.block_tokens;         // warp-uniform: block_tokens is a multiple of 32
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kTileExperts;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
+        const uint32_t t_zop = tmem_base + ((uint32_t)(q * 32) << 16) + kZopCol0 + acc * 64;
         bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
         if (ok) {
-            // ---- narrow z to [hi | lo] and store it as the K-major, 128-B-swizzled A operand
+            // ---- narrow z to bf16 [hi | lo] and store it to tensor memory as the A operand of phase 2
             tc_fence_after();
-            uint8_t* zrow = ring_ptr + acc * kZopOne + row_in_acc * 128;
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
@@ -373,38 +374,36 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
                     lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
                 }
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    // 16-byte chunk `ch` of the logical row [hi(RPAD) | lo(RPAD)]
-                    const int ch_hi = c * 2 + half, ch_lo = RPAD / 8 + c * 2 + half;
-                    const int slab_hi = ch_hi >> 3, slab_lo = ch_lo >> 3;
-                    uint4 vh = make_uint4(hi[half * 4], hi[half * 4 + 1], hi[half * 4 + 2], hi[half * 4 + 3]);
-                    uint4 vl = make_uint4(lo[half * 4], lo[half * 4 + 1], lo[half * 4 + 2], lo[half * 4 + 3]);
-                    *reinterpret_cast<uint4*>(zrow + slab_hi * 16384 + (((ch_hi & 7) ^ (row_in_acc & 7)) << 4)) = vh;
-                    *reinterpret_cast<uint4*>(zrow + slab_lo * 16384 + (((ch_lo & 7) ^ (row_in_acc & 7)) << 4)) = vl;
-                }
+                tmem_st8(t_zop + c * 8, hi);
+                tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
             }
-            fence_async_smem();
+            tmem_st_wait();
             tc_fence_before();
             mbar_arrive(bar(B_ZOP));
         }
 
         Selector<KCAP, kCandCap> S;
-        S.init(cand + row_in_blk * 8);
+        S.init(cand + row_in_blk * 16);
 #ifdef MORE_STATS
         unsigned st_chunks = 0, st_hit = 0, st_trip = 0, st_app = 0, st_rcall = 0, st_riter = 0, st_retry = 0, st_direct = 0;
+        (void)st_trip; (void)st_retry; (void)st_direct;
+        long long st_twait = 0, st_tproc = 0;
+        const long long st_t0 = clock64();
 #define STAT(x) x
 #else
 #define STAT(x)
 #endif
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
 
-        // `ok` is kept warp-uniform from here on (tcgen05.ld and the votes below need all 32 lanes).
+        // `ok` is kept warp-uniform from here on (tcgen05.ld, elect and the votes below need all 32 lanes).
         ok = __all_sync(kFullMask, ok);
-        for (int it = 0; it < ntiles && ok; ++it) {
-            const int e0 = (tile_lo + it) * kTileExperts;
-            const bool ragged = e0 + kTileExperts > p.M;
+
+        for (int it = 0; it < nsteps && ok; ++it) {
+            const int e0 = e_lo + it * kHalf;
+            const bool ragged = e0 + kHalf > p.M;
+            STAT(const long long tw0 = clock64();)
             ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
+            STAT(const long long tw1 = clock64(); st_twait += tw1 - tw0;)
             if (!ok) break;
             if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
                 mbar_arrive(bar(B_ACCE + acc));
@@ -415,7 +414,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             // in flight while the current 16 are processed.
             float va[16], vb[16];
             // ---- one 16-column chunk: triple maxima, optional online softmax update, candidate scan
-            auto process = [&](float (&v)[16], uint32_t ta, int col0) {
+            auto process = [&](float (&v)[16], int col0) {
                 if (ragged) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
@@ -424,7 +423,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 float t[5];
 #pragma unroll
                 for (int i = 0; i < 5; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                const float cmax = max3(max3(t[0], t[1], t[2]), max3(t[3], t[4], v[15]), -INFINITY);
+                const float cmax = fmaxf(max3(t[0], t[1], t[2]), max3(t[3], t[4], v[15]));
                 if (LSE) {
                     const float c2 = cmax * kLog2e;
                     if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
@@ -438,70 +437,37 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     }
                     zsum += (a0 + a1) + (a2 + a3);
                 }
-                // Append this chunk's candidates.  When some token of the warp runs out of buffer (always so on the
-                // very first chunk, when tau is -inf) the warp forgets the chunk's appends and folds the older
-                // candidates into the lists; with empty buffers and a fresher tau the chunk usually fits on a second
-                // scan, otherwise it is taken element by element, re-read from tensor memory.
-                STAT(st_chunks++; if (__any_sync(kFullMask, cmax > S.tau)) st_hit++;
-                     for (int i = 0; i < 5; ++i) if (__any_sync(kFullMask, t[i] > S.tau)) st_trip++;)
-                const uint32_t mark = S.ptr;
-                if (cmax > S.tau) S.scan(v, t, col0);
-                STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandSlotStride);)
-                bool direct = __any_sync(kFullMask, S.ptr >= S.lim);
-                if (direct) {
-                    S.ptr = mark;
-                    STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
-                    const bool had_older = __any_sync(kFullMask, mark != S.base);
-                    S.refresh();
-                    if (had_older) {
-                        STAT(st_retry++;)
-                        if (cmax > S.tau) S.scan(v, t, col0);
-                        direct = __any_sync(kFullMask, S.ptr >= S.lim);
-                        if (direct) S.ptr = S.base;
+                // Append this chunk's candidate groups (a warp-uniform branch around predicated stores), then fold
+                // the buffers into the lists if some token of the warp is running out of slots.
+                STAT(st_chunks++;)
+                if (__any_sync(kFullMask, cmax > S.tau)) {
+                    STAT(st_hit++; const uint32_t mark = S.ptr;)
+                    S.scan(v, t, col0);
+                    STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandSlotStride);)
+                    if (__any_sync(kFullMask, S.ptr >= S.warn)) {
+                        STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
+                        S.refresh();
                     }
-                }
-                if (direct) {
-#pragma unroll 1
-                    for (int g = 0; g < 2; ++g) {
-                        uint32_t xb[8];
-                        asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                                     : "=r"(xb[0]), "=r"(xb[1]), "=r"(xb[2]), "=r"(xb[3]), "=r"(xb[4]), "=r"(xb[5]),
-                                       "=r"(xb[6]), "=r"(xb[7])
-                                     : "r"(ta + g * 8)
-                                     : "memory");
-                        asm volatile("tcgen05.wait::ld.sync.aligned;"
-                                     : "+r"(xb[0]), "+r"(xb[1]), "+r"(xb[2]), "+r"(xb[3]), "+r"(xb[4]), "+r"(xb[5]),
-                                       "+r"(xb[6]), "+r"(xb[7])::"memory");
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) {
-                            const float x = __uint_as_float(xb[i]);
-                            const int cj = col0 + g * 8 + i;
-                            if (cj < p.M && x > S.L.tau()) S.L.insert(x, cj);
-                        }
-                    }
-                    S.tau = S.L.tau();
-                    STAT(st_direct++;)
                 }
             };
+            // columns 0-31: the load of the next 16 columns is in flight while the current 16 are processed
             tmem_ld16(t_lane, va);
-#pragma unroll 1
-            for (int c = 0; c < kTileExperts / 32; ++c) {
-                const uint32_t ta = t_lane + c * 32;
-                const int col0 = e0 + c * 32;
-                tmem_ld_wait16(va);
-                tmem_ld16(ta + 16, vb);
-                process(va, ta, col0);
-                // (a direct-mode re-read inside process waits for all loads, including the one just issued: harmless)
-                tmem_ld_wait16(vb);
-                if (c + 1 < kTileExperts / 32) tmem_ld16(ta + 32, va);
-                process(vb, ta + 16, col0 + 16);
-            }
+            tmem_ld_wait16(va);
+            tmem_ld16(t_lane + 16, vb);
+            process(va, e0);
+            tmem_ld_wait16(vb);
+            tmem_ld16(t_lane + 32, va);
+            process(vb, e0 + 16);
+            // columns 32-63: both halves are brought into registers first; the accumulator can then be handed back,
+            // and the next step's MMAs run while these 32 columns are processed
+            tmem_ld_wait16(va);
+            tmem_ld16(t_lane + 48, vb);
+            tmem_ld_wait16(vb);
             tc_fence_before();
-            mbar_arrive(bar(B_ACCE + acc));                  // this accumulator may be overwritten now
-            if (__any_sync(kFullMask, S.ptr >= S.warn)) {
-                STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
-                S.refresh();
-            }
+            mbar_arrive(bar(B_ACCE + acc));
+            process(va, e0 + 32);
+            process(vb, e0 + 48);
+            STAT(st_tproc += clock64() - tw1;)
         }
         S.refresh();
         TopList<KCAP>& L = S.L;
@@ -515,6 +481,10 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             atomicAdd(p.stats + 5, (unsigned long long)st_riter);
             atomicAdd(p.stats + 6, (unsigned long long)st_retry);
             atomicAdd(p.stats + 7, (unsigned long long)st_direct);
+            atomicAdd(p.stats + 8, (unsigned long long)st_twait);
+            atomicAdd(p.stats + 9, (unsigned long long)st_tproc);
+            atomicAdd(p.stats + 10, (unsigned long long)(clock64() - st_t0));
+            atomicAdd(p.stats + 11, 1ull);
         }
 #endif
 

@@ -21,7 +21,7 @@ constexpr int kP1StageBytes = kXTileBytes + kR1TileBytes;
 constexpr int kRingBytes = 110 * 1024;             // phase 1: the two stages; phase 2: A operands, candidates, R2 stages
 static_assert(kStagesP1 * kP1StageBytes <= kRingBytes, "phase-1 ring does not fit");
 constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
-constexpr int kTmemCols = 256;                     // two 128-token x 128-expert fp32 accumulators
+constexpr int kTmemCols = 256;                     // tensor-memory columns per CTA (two CTAs share the 512 of an SM)
 constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s
 constexpr uint32_t kSuspendHintNs = 20000;              // a waiting thread may be parked this long per try
 
@@ -99,6 +99,65 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, ui
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+
+// Same, with the A operand read from tensor memory: lane = row of A, each 32-bit column holds two consecutive
+// bf16 K-elements (the lower index in the lower half), so one K = 16 step spans 8 columns.
+__device__ __forceinline__ void tc_mma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+// Warp-converged issue: all 32 lanes of the issuing warp execute these; elect.sync picks the one lane (the same on
+// every call) that issues the instruction.  Keeping the warp converged and passing the shared-memory descriptors as
+// two 32-bit words (low word = start address, advanced with one integer add per K step) keeps the issuing code short
+// enough that it does not limit the tensor pipe: with descriptors rebuilt per instruction inside a one-lane branch
+// the issue alone took 50-80 clocks per instruction, more than the 32 clocks a 128 x 64 x 16 MMA computes for.
+__device__ __forceinline__ void tc_mma_bf16_ts_elect(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi,
+                                                     uint32_t idesc, bool accumulate)
+{
+    if (accumulate)
+        asm volatile(
+            "{\n\t.reg .pred p, pe;\n\t.reg .b64 bd;\n\t"
+            "setp.eq.u32 p, 0, 0;\n\tmov.b64 bd, {%2, %3};\n\telect.sync _|pe, 0xffffffff;\n\t"
+            "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else
+        asm volatile(
+            "{\n\t.reg .pred p, pe;\n\t.reg .b64 bd;\n\t"
+            "setp.ne.u32 p, 0, 0;\n\tmov.b64 bd, {%2, %3};\n\telect.sync _|pe, 0xffffffff;\n\t"
+            "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], bd, %4, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16_ss_elect(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo,
+                                                     uint32_t b_hi, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, pe;\n\t.reg .b64 ad, bd;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\tmov.b64 ad, {%1, %2};\n\tmov.b64 bd, {%3, %4};\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tc_commit_elect(uint32_t bar)
+{
+    asm volatile(
+        "{\n\t.reg .pred pe;\n\telect.sync _|pe, 0xffffffff;\n\t"
+        "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
+}
+
+// Store 8 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&u)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                 ::"r"(taddr), "r"(u[0]), "r"(u[1]), "r"(u[2]), "r"(u[3]), "r"(u[4]), "r"(u[5]), "r"(u[6]), "r"(u[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // 16 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16])
