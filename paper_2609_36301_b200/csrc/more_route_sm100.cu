@@ -33,6 +33,13 @@
 
 #include <limits.h>
 
+// -DMORE_STATS builds count epilogue events and clocks into KernelParams::stats (diagnostics only).
+#ifdef MORE_STATS
+#define STAT(...) __VA_ARGS__
+#else
+#define STAT(...)
+#endif
+
 namespace more {
 
 namespace {
@@ -80,77 +87,94 @@ struct TopList {
 };
 
 // Running top-k of one token.  Between refreshes the sorted list is left alone.  A chunk of 16 logits is looked at
-// as five triples and a single; every group whose maximum beats the cached threshold `tau` (the list's last entry
-// as of the last refresh, hence never above the true threshold) is appended whole, in ascending column order, to
-// this thread's column of a shared-memory candidate buffer: one predicated 16-byte store {v0, v1, v2, first column}
-// and no branch.  refresh() then inserts the buffered elements that beat the up-to-date threshold, so the inserts of
-// several chunks of all 32 tokens of a warp are executed together.  A chunk appends at most 6 entries and the warp
-// refreshes as soon as some token has fewer than 6 free slots left, so the buffer cannot overflow.
-constexpr int kCandSlotStride = kEpilogueThreads * 16;    // bytes between successive slots of one thread
+// as four groups of four; every group whose maximum beats the cached threshold `tau` (the list's last entry as of
+// the last refresh, hence never above the true threshold) is appended whole, in ascending column order, to this
+// thread's column of a shared-memory candidate buffer: one predicated 16-byte store of the four values (they sit in
+// four consecutive registers as loaded from tensor memory, so nothing is moved), one predicated 4-byte store of the
+// group's first column into a parallel array, and no branch.  refresh() then inserts the buffered elements that beat
+// the up-to-date threshold, so the inserts of several chunks of all 32 tokens of a warp are executed together.  A
+// chunk appends at most 4 entries and the warp refreshes as soon as some token has fewer than 4 free slots left, so
+// the buffer cannot overflow.
+constexpr int kCandValStride = kEpilogueThreads * 16;     // bytes between successive value slots of one thread
+constexpr int kCandColStride = kEpilogueThreads * 4;      // ... and between its column slots
 #ifndef MORE_CAND_CAP
-#define MORE_CAND_CAP 14
+#define MORE_CAND_CAP 12
 #endif
 #ifndef MORE_WARN
-#define MORE_WARN (MORE_CAND_CAP - 6)
+#define MORE_WARN (MORE_CAND_CAP - 4)
 #endif
-static_assert(MORE_WARN >= 1 && MORE_WARN <= MORE_CAND_CAP - 6, "a chunk must always find 6 free slots");
+static_assert(MORE_WARN >= 1 && MORE_WARN <= MORE_CAND_CAP - 4, "a chunk must always find 4 free slots");
 constexpr unsigned kFullMask = 0xffffffffu;
 
 template <int KCAP, int CAP>
 struct Selector {
     TopList<KCAP> L;
     float tau;
-    uint32_t ptr;     // shared-memory address of this thread's next free candidate slot
-    uint32_t base;    // its first slot
+    uint32_t ptr;     // shared-memory address of this thread's next free value slot
+    uint32_t cptr;    // ... and of the matching column slot
+    uint32_t base, cbase;
     uint32_t warn;    // at or beyond this fill level the warp refreshes after the chunk
 
-    __device__ __forceinline__ void init(uint32_t first_slot)
+    __device__ __forceinline__ void init(uint32_t first_val_slot, uint32_t first_col_slot)
     {
         L.init();
         tau = -INFINITY;
-        base = ptr = first_slot;
-        warn = first_slot + MORE_WARN * kCandSlotStride;
+        base = ptr = first_val_slot;
+        cbase = cptr = first_col_slot;
+        warn = first_val_slot + MORE_WARN * kCandValStride;
     }
+    // Called by all 32 lanes of a warp together.  Every round inserts at most one element per token: the maximum
+    // of the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
+    // (rising) threshold any more moves on to its next entries.  The rounds end when no token has anything left, so
+    // their number is the largest count of real insertions of any token of the warp, and the (select-only) insert
+    // code is executed once per round.
     __device__ __forceinline__ void refresh()
     {
-        for (uint32_t a = base; a < ptr; a += kCandSlotStride) {
-            float x0, x1, x2;
-            int col;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=r"(col) : "r"(a) : "memory");
-            const float m = max3(x0, x1, x2);
-            if (m > L.tau()) {
-                // the group's maximum first (its lowest column on a tie), then, rarely, the other two in column order
-                const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : 2);
-                L.insert(m, col + j);
-                const float y0 = (j == 0) ? x1 : x0, y1 = (j == 2) ? x1 : x2;
-                const int c0 = col + ((j == 0) ? 1 : 0), c1 = col + ((j == 2) ? 1 : 2);
-                if (fmaxf(y0, y1) > L.tau()) {
-                    if (y0 > L.tau()) L.insert(y0, c0);
-                    if (y1 > L.tau()) L.insert(y1, c1);
-                }
+        uint32_t a = base, c = cbase;
+        float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
+        int col = 0;
+        for (;;) {
+            float m = fmaxf(max3(x0, x1, x2), x3);
+            while (!(m > L.tau()) && a < ptr) {
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(a) : "memory");
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(col) : "r"(c) : "memory");
+                a += kCandValStride;
+                c += kCandColStride;
+                m = fmaxf(max3(x0, x1, x2), x3);
             }
+            const bool pass = m > L.tau();
+            if (!__any_sync(kFullMask, pass)) break;
+            // the maximum's lowest column on a tie, so that equal logits enter the list in ascending column order
+            const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : ((x2 == m) ? 2 : 3));
+            if (pass) L.insert(m, col + j);
+            x0 = (j == 0) ? -INFINITY : x0;
+            x1 = (j == 1) ? -INFINITY : x1;
+            x2 = (j == 2) ? -INFINITY : x2;
+            x3 = (j == 3) ? -INFINITY : x3;
         }
         ptr = base;
+        cptr = cbase;
         tau = L.tau();
     }
-    // if (t > tau) append {v0, v1, v2, col}
-    __device__ __forceinline__ void append3(float t, float v0, float v1, float v2, int col)
+    // if (t > tau) append {v0, v1, v2, v3} and col
+    __device__ __forceinline__ void append4(float t, float v0, float v1, float v2, float v3, int col)
     {
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "setp.gt.f32 p, %1, %6;\n\t"
-            "@p st.shared.v4.b32 [%0], {%2, %3, %4, %5};\n\t"
-            "@p add.u32 %0, %0, %7;\n\t}"
-            : "+r"(ptr)
-            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "r"(col), "f"(tau), "n"(kCandSlotStride)
+            "setp.gt.f32 p, %2, %8;\n\t"
+            "@p st.shared.v4.b32 [%0], {%3, %4, %5, %6};\n\t"
+            "@p st.shared.b32 [%1], %7;\n\t"
+            "@p add.u32 %0, %0, %9;\n\t"
+            "@p add.u32 %1, %1, %10;\n\t}"
+            : "+r"(ptr), "+r"(cptr)
+            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "f"(v3), "r"(col), "f"(tau), "n"(kCandValStride), "n"(kCandColStride)
             : "memory");
     }
-    // v: 16 logits of columns col0.., t: maxima of the triples (v[3i], v[3i+1], v[3i+2]) for i < 5; v[15] stands alone.
-    __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[5], int col0)
+    // v: 16 logits of columns col0.., t: maxima of the groups (v[4i] .. v[4i+3]).
+    __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[4], int col0)
     {
 #pragma unroll
-        for (int i = 0; i < 5; ++i) append3(t[i], v[3 * i], v[3 * i + 1], v[3 * i + 2], col0 + 3 * i);
-        append3(v[15], v[15], -INFINITY, -INFINITY, col0 + 15);
+        for (int i = 0; i < 4; ++i) append4(t[i], v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3], col0 + 4 * i);
     }
 };
 
@@ -213,7 +237,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
     constexpr int kStagesP2 = (RPAD == 64) ? 6 : 8;             // R2 blocks in flight
     constexpr int kCandCap = MORE_CAND_CAP;                     // candidate slots per token
-    constexpr int kCandBytes = kCandCap * kCandSlotStride;
+    constexpr int kCandValBytes = kCandCap * kCandValStride;
+    constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);
     static_assert(kCandBytes + kStagesP2 * kR2StageBytes <= kRingBytes, "phase-2 layout does not fit");
     // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
     // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.
@@ -236,6 +261,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
+    STAT(const long long st_top = clock64();)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int blk = blockIdx.x / p.msplit, split = blockIdx.x % p.msplit;
     const int tok0 = blk * p.block_tokens;
@@ -356,7 +382,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const bool warp_live = acc * 128 + q * 32 < p.block_tokens;         // warp-uniform: block_tokens is a multiple of 32
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
         const uint32_t t_zop = tmem_base + ((uint32_t)(q * 32) << 16) + kZopCol0 + acc * 64;
+        STAT(const long long st_k0 = clock64();)
         bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
+        STAT(const long long st_k1 = clock64();)
         if (ok) {
             // ---- narrow z to bf16 [hi | lo] and store it to tensor memory as the A operand of phase 2
             tc_fence_after();
@@ -383,16 +411,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         }
 
         Selector<KCAP, kCandCap> S;
-        S.init(cand + row_in_blk * 16);
-#ifdef MORE_STATS
-        unsigned st_chunks = 0, st_hit = 0, st_trip = 0, st_app = 0, st_rcall = 0, st_riter = 0, st_retry = 0, st_direct = 0;
-        (void)st_trip; (void)st_retry; (void)st_direct;
-        long long st_twait = 0, st_tproc = 0;
-        const long long st_t0 = clock64();
-#define STAT(x) x
-#else
-#define STAT(x)
-#endif
+        S.init(cand + row_in_blk * 16, cand + kCandValBytes + row_in_blk * 4);
+        STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_rcall = 0, st_riter = 0; long long st_twait = 0, st_tproc = 0, st_tref = 0;
+             const long long st_t0 = clock64();)
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
 
         // `ok` is kept warp-uniform from here on (tcgen05.ld, elect and the votes below need all 32 lanes).
@@ -401,29 +422,21 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         for (int it = 0; it < nsteps && ok; ++it) {
             const int e0 = e_lo + it * kHalf;
             const bool ragged = e0 + kHalf > p.M;
-            STAT(const long long tw0 = clock64();)
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
-            STAT(const long long tw1 = clock64(); st_twait += tw1 - tw0;)
-            if (!ok) break;
-            if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
-                mbar_arrive(bar(B_ACCE + acc));
-                continue;
-            }
-            tc_fence_after();
-            // The tile is read 16 columns at a time into two register buffers: the load of the next 16 columns is
-            // in flight while the current 16 are processed.
             float va[16], vb[16];
             // ---- one 16-column chunk: triple maxima, optional online softmax update, candidate scan
             auto process = [&](float (&v)[16], int col0) {
+#ifdef MORE_EXP_NOPROC
+                return;
+#endif
                 if (ragged) {
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
                         if (col0 + i >= p.M) v[i] = -INFINITY;
                 }
-                float t[5];
+                float t[4];
 #pragma unroll
-                for (int i = 0; i < 5; ++i) t[i] = max3(v[3 * i], v[3 * i + 1], v[3 * i + 2]);
-                const float cmax = fmaxf(max3(t[0], t[1], t[2]), max3(t[3], t[4], v[15]));
+                for (int i = 0; i < 4; ++i) t[i] = fmaxf(max3(v[4 * i], v[4 * i + 1], v[4 * i + 2]), v[4 * i + 3]);
+                const float cmax = fmaxf(max3(t[0], t[1], t[2]), t[3]);
                 if (LSE) {
                     const float c2 = cmax * kLog2e;
                     if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
@@ -440,16 +453,32 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 // Append this chunk's candidate groups (a warp-uniform branch around predicated stores), then fold
                 // the buffers into the lists if some token of the warp is running out of slots.
                 STAT(st_chunks++;)
+#ifdef MORE_EXP_NOSCAN
+                m2 = fmaxf(m2, cmax);
+                return;
+#endif
                 if (__any_sync(kFullMask, cmax > S.tau)) {
                     STAT(st_hit++; const uint32_t mark = S.ptr;)
                     S.scan(v, t, col0);
-                    STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandSlotStride);)
-                    if (__any_sync(kFullMask, S.ptr >= S.warn)) {
-                        STAT(st_rcall++; st_riter += __reduce_max_sync(kFullMask, (S.ptr - S.base) / kCandSlotStride);)
+                    STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
+                    const uint32_t fill = __reduce_max_sync(kFullMask, S.ptr - S.base);
+                    if (fill >= MORE_WARN * kCandValStride) {
+                        // some token is about to run out of slots: fold now
+                        STAT(st_rcall++; st_riter += fill / kCandValStride; const long long tr0 = clock64();)
                         S.refresh();
+                        STAT(st_tref += clock64() - tr0;)
                     }
                 }
             };
+            STAT(const long long tw0 = clock64();)
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
+            STAT(const long long tw1 = clock64(); st_twait += tw1 - tw0;)
+            if (!ok) break;
+            if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
+                mbar_arrive(bar(B_ACCE + acc));
+                continue;
+            }
+            tc_fence_after();
             // columns 0-31: the load of the next 16 columns is in flight while the current 16 are processed
             tmem_ld16(t_lane, va);
             tmem_ld_wait16(va);
@@ -475,16 +504,17 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         if (lane == 0 && p.stats) {
             atomicAdd(p.stats + 0, (unsigned long long)st_chunks);
             atomicAdd(p.stats + 1, (unsigned long long)st_hit);
-            atomicAdd(p.stats + 2, (unsigned long long)st_trip);
             atomicAdd(p.stats + 3, (unsigned long long)st_app);
             atomicAdd(p.stats + 4, (unsigned long long)st_rcall);
             atomicAdd(p.stats + 5, (unsigned long long)st_riter);
-            atomicAdd(p.stats + 6, (unsigned long long)st_retry);
-            atomicAdd(p.stats + 7, (unsigned long long)st_direct);
             atomicAdd(p.stats + 8, (unsigned long long)st_twait);
             atomicAdd(p.stats + 9, (unsigned long long)st_tproc);
             atomicAdd(p.stats + 10, (unsigned long long)(clock64() - st_t0));
             atomicAdd(p.stats + 11, 1ull);
+            atomicAdd(p.stats + 12, (unsigned long long)st_tref);
+            atomicAdd(p.stats + 13, (unsigned long long)(st_k1 - st_k0));
+            atomicAdd(p.stats + 14, (unsigned long long)(st_t0 - st_k1));
+            atomicAdd(p.stats + 2, (unsigned long long)(st_k0 - st_top));
         }
 #endif
 
@@ -563,6 +593,11 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // ---- common exit: everyone arrives here, also after an abort
     tc_fence_before();
     __syncthreads();
+    STAT(if (threadIdx.x == 64 && p.stats) {
+        atomicAdd(p.stats + 6, (unsigned long long)(clock64() - st_top));      // CTA lifetime, clk
+        atomicMax(p.stats + 7, (unsigned long long)(clock64() - st_top));      // longest CTA
+        atomicAdd(p.stats + 15, 1ull);
+    })
     if (*abort_flag && threadIdx.x == 0) {
         // give bulk copies that may still be in flight time to land before shared memory is released
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
