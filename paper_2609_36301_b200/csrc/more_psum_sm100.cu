@@ -113,55 +113,59 @@ psum_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         }
     } else if (warp == 1) {
         // ======================================================================================= MMA issuer
-        if (lane == 0) {
-            bool ok = true;
-            constexpr uint32_t idesc1 = umma_idesc(64);
-            // second contraction transposed: A = R2 tile (MN-major), B = z operand (K-major), 128 experts x 128 tokens
-            constexpr uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
-                                        ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        // The whole warp runs this code converged and one elected lane issues each instruction; the descriptors are
+        // words computed once plus integer offsets (see tc_mma_bf16_ss_elect).
+        constexpr unsigned kFull = 0xffffffffu;
+        bool ok = true;
+        constexpr uint32_t idesc1 = umma_idesc(64);
+        // second contraction transposed: A = R2 tile (MN-major), B = z operand (K-major), 128 experts x 128 tokens
+        constexpr uint32_t idesc2 = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | (0u << 16) |
+                                    ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+        {
+            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
+            const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
                 const int s = kt % kStagesP1;
-                ok = mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status);
+                ok = __all_sync(kFull, mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t xa = ring + s * kP1StageBytes, rb = xa + kXTileBytes;
+                const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), r_lo = r_lo0 + s * (kP1StageBytes >> 4);
 #pragma unroll
                 for (int a = 0; a < 2; ++a) {
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t ad = umma_desc_sw128(xa + a * 16384 + kk * 32, 16, 1024);
-                        const uint64_t bd = umma_desc_sw128(rb + kk * 2048, 8192, 1024);
-                        tc_mma_bf16(tmem_base + a * kTileExperts, ad, bd, idesc1, (kt | kk) != 0);
-                    }
+                    for (int kk = 0; kk < 4; ++kk)
+                        tc_mma_bf16_ss_elect(tmem_base + a * kTileExperts, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
+                                             r_lo + kk * (2048 >> 4), r_hi, idesc1, (kt | kk) != 0);
                 }
-                tc_commit(bar(B_EMPTY1 + s));
+                tc_commit_elect(bar(B_EMPTY1 + s));
             }
-            if (ok) tc_commit(bar(B_ZACC));
-            ok = ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status);
-            tc_fence_after();
-            for (int it = 0; it < ntiles && ok; ++it) {
-                const int s = it % kStagesP2;
-                ok = mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status);
+        }
+        if (ok) tc_commit_elect(bar(B_ZACC));
+        ok = __all_sync(kFull, ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status));
+        tc_fence_after();
+        const uint64_t ad0 = umma_desc_sw128(r2ring, RPAD * 128, 1024), zd0 = umma_desc_sw128(zop, 16, 1024);
+        const uint32_t a_lo0 = (uint32_t)ad0, a_hi = (uint32_t)(ad0 >> 32), z_lo0 = (uint32_t)zd0, z_hi = (uint32_t)(zd0 >> 32);
+        for (int it = 0; it < ntiles && ok; ++it) {
+            const int s = it % kStagesP2;
+            ok = __all_sync(kFull, mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status));
+            if (!ok) break;
+            const uint32_t a_lo = a_lo0 + s * (kR2StageBytes >> 4);
+#pragma unroll
+            for (int a = 0; a < 2; ++a) {            // token half a -> TMEM columns a*128 ..
+                ok = __all_sync(kFull, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
                 if (!ok) break;
-                const uint32_t rb = r2ring + s * kR2StageBytes;
+                tc_fence_after();
 #pragma unroll
-                for (int a = 0; a < 2; ++a) {            // token half a -> TMEM columns a*128 ..
-                    ok = ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll
-                    for (int j = 0; j < 2 * kKSteps; ++j) {
-                        const uint32_t zbyte = j * 32;                                       // K offset in [hi | lo]
-                        const uint64_t ad = umma_desc_sw128(rb + (j % kKSteps) * 2048, RPAD * 128, 1024);
-                        const uint64_t bd =
-                            umma_desc_sw128(zop + a * kZopOne + (zbyte >> 7) * 16384 + (zbyte & 127), 16, 1024);
-                        tc_mma_bf16(tmem_base + a * 128, ad, bd, idesc2, j != 0);
-                    }
-                    tc_commit(bar(B_ACCF + a));
+                for (int j = 0; j < 2 * kKSteps; ++j) {
+                    const uint32_t zbyte = j * 32;                                       // K offset in [hi | lo]
+                    tc_mma_bf16_ss_elect(tmem_base + a * 128, a_lo + (j % kKSteps) * (2048 >> 4), a_hi,
+                                         z_lo0 + ((a * kZopOne + (zbyte >> 7) * 16384 + (zbyte & 127)) >> 4), z_hi, idesc2,
+                                         j != 0);
                 }
-                if (!ok) break;
-                tc_commit(bar(B_EMPTY2 + s));
+                tc_commit_elect(bar(B_ACCF + a));
             }
+            if (!ok) break;
+            tc_commit_elect(bar(B_EMPTY2 + s));
         }
     } else {
         // ========================================================================================= epilogue
