@@ -27,10 +27,11 @@ class MoreRouteError(RuntimeError):
 
 
 def lib() -> ctypes.CDLL:
-    """Load (once) the in-tree shared library; raises if it has not been built."""
+    """Load (once) the in-tree shared library; raises if it has not been built.  ``MORE_ROUTE_LIB`` names another
+    build of the same sources to load instead (the diagnostic builds of ``build.py``)."""
     global _lib
     if _lib is None:
-        path = _build.LIB_PATH
+        path = os.environ.get("MORE_ROUTE_LIB") or _build.LIB_PATH
         if not os.path.exists(path):
             raise FileNotFoundError(
                 f"{path} is missing: build it with `python -m paper_2609_36301_b200.build` "

@@ -19,16 +19,28 @@ def _newest_source_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the CUDA sources if the library is missing or older than any source; return its path."""
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _newest_source_mtime():
-        return LIB_PATH
+def build(force: bool = False, verbose: bool = False, out: str | None = None, defines: tuple = ()) -> str:
+    """Compile the CUDA sources if the library is missing or older than any source; return its path.
+
+    ``defines`` adds ``-D`` switches (the diagnostic builds: ``MORE_STATS`` for event and clock counters,
+    ``MORE_EXP_NOSCAN`` / ``MORE_EXP_NOPROC`` for the epilogue with its candidate handling, or everything but the
+    tensor-memory loads, compiled out); such a build goes to ``out``, never over the product library."""
+    target = out or LIB_PATH
+    if defines and target == LIB_PATH:
+        raise ValueError("a diagnostic build needs its own output path")
+    if not force and os.path.exists(target) and os.path.getmtime(target) >= _newest_source_mtime():
+        return target
     nvcc = os.environ.get("NVCC", "nvcc")
-    cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", LIB_PATH] + \
-          [os.path.join(_CSRC, s) for s in SOURCES]
+    cmd = [nvcc] + NVCC_FLAGS + ["-D" + d for d in defines] + (["-Xptxas", "-v"] if verbose else []) + \
+          ["-o", target] + [os.path.join(_CSRC, s) for s in SOURCES]
     subprocess.run(cmd, check=True)
-    return LIB_PATH
+    return target
 
 
 if __name__ == "__main__":
-    print(build(force=True, verbose=True))
+    import sys
+    # python -m paper_2609_36301_b200.build [OUT.so DEFINE ...]
+    if len(sys.argv) > 2:
+        print(build(force=True, out=sys.argv[1], defines=tuple(sys.argv[2:])))
+    else:
+        print(build(force=True, verbose=True))
