@@ -358,6 +358,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const uint32_t b_lo = b_lo0 + s * (kR2StageBytes >> 4);
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
+                if (a * 128 >= p.block_tokens) continue;     // a group without tokens takes no part in phase 2
                 // accumulator a is free once its 128 epilogue threads have read the previous step out of it
                 ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
                 if (!ok) break;
@@ -419,7 +420,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // `ok` is kept warp-uniform from here on (tcgen05.ld, elect and the votes below need all 32 lanes).
         ok = __all_sync(kFullMask, ok);
 
-        for (int it = 0; it < nsteps && ok; ++it) {
+        const bool group_live = acc * 128 < p.block_tokens;
+        for (int it = 0; it < nsteps && ok && group_live; ++it) {
             const int e0 = e_lo + it * kHalf;
             const bool ragged = e0 + kHalf > p.M;
             float va[16], vb[16];
