@@ -48,6 +48,9 @@ def _load():
         lib.more_oracle_psum.restype = ctypes.c_int
         lib.more_oracle_dispatch.argtypes = [i32p, ctypes.c_int64, ctypes.c_int, ctypes.c_int, i64p, i64p]
         lib.more_oracle_dispatch.restype = ctypes.c_int
+        lib.more_oracle_merge.argtypes = [i32p, f64p, f64p, ctypes.c_int, ctypes.c_int64, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_int, i32p, f64p, f64p, f64p, i64p]
+        lib.more_oracle_merge.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -153,3 +156,29 @@ def psum(X, R1, R2):
     if rc != 0:
         raise ValueError("more_oracle_psum rejected its arguments")
     return out, lse
+
+
+def merge(idx, val, lse, M: int, gate_mode: int):
+    """Global top-k from per-shard top-k lists: ``idx [S][T][k]`` (global expert ids, < 0 = unused), ``val [S][T][k]``,
+    ``lse [S][T]`` or None.  Returns ``(idx [T][k], gate [T][k], val [T][k], lse [T] or None, counts [M])``."""
+    lib = _load()
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    val = np.ascontiguousarray(val, dtype=np.float64)
+    S, T, k = idx.shape
+    if val.shape != idx.shape:
+        raise ValueError("idx and val must have the same shape")
+    lse_c = None if lse is None else np.ascontiguousarray(lse, dtype=np.float64)
+    if lse_c is not None and lse_c.shape != (S, T):
+        raise ValueError("lse must be [S][T]")
+    out_idx = np.zeros((T, k), dtype=np.int32)
+    out_gate = np.zeros((T, k), dtype=np.float64)
+    out_val = np.zeros((T, k), dtype=np.float64)
+    out_lse = np.zeros((T,), dtype=np.float64) if lse_c is not None else None
+    counts = np.zeros((M,), dtype=np.int64)
+    rc = lib.more_oracle_merge(_p(idx, ctypes.c_int32), _p(val, ctypes.c_double),
+                               None if lse_c is None else _p(lse_c, ctypes.c_double), S, T, k, M, gate_mode,
+                               _p(out_idx, ctypes.c_int32), _p(out_gate, ctypes.c_double), _p(out_val, ctypes.c_double),
+                               None if out_lse is None else _p(out_lse, ctypes.c_double), _p(counts, ctypes.c_int64))
+    if rc != 0:
+        raise ValueError("more_oracle_merge rejected its arguments")
+    return out_idx, out_gate, out_val, out_lse, counts

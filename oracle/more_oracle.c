@@ -23,7 +23,8 @@
  *
  * Pins (tests/test_oracle_pins.py): numpy brute force on tiny inputs, the Thm. 1 basis construction, the
  * Prop. 1 sign-vector router (closed-form top-2, uniform marginals), the full-rank identity R1 = I, the
- * online-softmax recurrence Eq. app_online, permutation equivariance, and structural invariants.
+ * online-softmax recurrence Eq. app_online, permutation equivariance, and structural invariants; the shard merge
+ * (more_oracle_merge) against the unsharded route on every split of the experts tried.
  * On the large benchmark configurations nothing other than these pins fixes the values: parity unpinned there.
  */
 #include <math.h>
@@ -247,5 +248,76 @@ int more_oracle_psum(const uint16_t* X, const uint16_t* R1, const uint16_t* R2,
         if (lse) lse[n] = m + log(Z);
     }
     free(R1d); free(R2d); free(z); free(l);
+    return 0;
+}
+
+/*
+ * Hierarchical top-k over an expert dimension that is split into S shards (the paper's remark that a router sharded
+ * over devices needs a local top-k per shard followed by a global top-k; the merge of the online-softmax pair is
+ * Eq. app_online applied to whole shards).  Every shard s has routed the same T tokens over its own experts and
+ * reports, per token, its k best (global expert id, logit) pairs in any order (id < 0 marks an unused slot) and,
+ * optionally, lse_s = log sum_{i in shard} exp(l_i).  Plain definition: the union of the S*k pairs is sorted by
+ * (logit descending, id ascending) and its first k entries are the answer -- an expert outside its own shard's top
+ * k cannot be in the global top k.  lse = log sum_s exp(lse_s).  Gates as in more_oracle_route: softmax over the k
+ * selected logits (gate_mode 0) or exp(l - lse) (gate_mode 1, needs lse).  counts = histogram of the chosen ids.
+ *   idx [S][T][k], val [S][T][k], lse_in [S][T] or NULL; out_idx [T][k], out_gate [T][k], out_val [T][k] (may be NULL),
+ *   out_lse [T] (may be NULL), out_counts [M].  A token with fewer than k valid pairs gets id -1 / gate 0 in the
+ *   unused places.
+ */
+int more_oracle_merge(const int32_t* idx, const double* val, const double* lse_in, int S, int64_t T, int k, int M,
+                      int gate_mode, int32_t* out_idx, double* out_gate, double* out_val, double* out_lse,
+                      int64_t* out_counts)
+{
+    if (S < 1 || T < 0 || k < 1 || M < 1 || !idx || !val || !out_idx || !out_gate || !out_counts) return -1;
+    if (gate_mode != 0 && gate_mode != 1) return -1;
+    if (gate_mode == 1 && !lse_in) return -1;
+    const int n = S * k;
+    int32_t* ci = (int32_t*)malloc((size_t)n * sizeof(int32_t));
+    double* cv = (double*)malloc((size_t)n * sizeof(double));
+    if (!ci || !cv) { free(ci); free(cv); return -1; }
+    for (int e = 0; e < M; ++e) out_counts[e] = 0;
+    for (int64_t t = 0; t < T; ++t) {
+        int c = 0;
+        for (int s = 0; s < S; ++s)
+            for (int j = 0; j < k; ++j) {
+                const size_t p = ((size_t)s * (size_t)T + (size_t)t) * (size_t)k + (size_t)j;
+                if (idx[p] >= 0 && idx[p] < M) { ci[c] = idx[p]; cv[c] = val[p]; ++c; }
+            }
+        /* selection sort of the first k places by (value desc, id asc) */
+        const int kk = c < k ? c : k;
+        for (int a = 0; a < kk; ++a) {
+            int best = a;
+            for (int b = a + 1; b < c; ++b)
+                if (cv[b] > cv[best] || (cv[b] == cv[best] && ci[b] < ci[best])) best = b;
+            const int32_t ti = ci[a]; ci[a] = ci[best]; ci[best] = ti;
+            const double tv = cv[a]; cv[a] = cv[best]; cv[best] = tv;
+        }
+        double lse = 0.0;
+        if (lse_in) {
+            double m = -INFINITY;
+            for (int s = 0; s < S; ++s) if (lse_in[(size_t)s * (size_t)T + (size_t)t] > m) m = lse_in[(size_t)s * (size_t)T + (size_t)t];
+            double z = 0.0;
+            for (int s = 0; s < S; ++s) z += exp(lse_in[(size_t)s * (size_t)T + (size_t)t] - m);
+            lse = m + log(z);
+            if (out_lse) out_lse[t] = lse;
+        }
+        double denom = 0.0;
+        if (gate_mode == 0)
+            for (int a = 0; a < kk; ++a) denom += exp(cv[a] - cv[0]);
+        for (int a = 0; a < k; ++a) {
+            const size_t o = (size_t)t * (size_t)k + (size_t)a;
+            if (a < kk) {
+                out_idx[o] = ci[a];
+                out_gate[o] = gate_mode == 0 ? exp(cv[a] - cv[0]) / denom : exp(cv[a] - lse);
+                if (out_val) out_val[o] = cv[a];
+                out_counts[ci[a]] += 1;
+            } else {
+                out_idx[o] = -1;
+                out_gate[o] = 0.0;
+                if (out_val) out_val[o] = -INFINITY;
+            }
+        }
+    }
+    free(ci); free(cv);
     return 0;
 }

@@ -300,3 +300,56 @@ def test_psum_is_equivariant_under_expert_relabelling():
     a, _ = oracle.psum(case.X, case.R1, case.R2)
     b, _ = oracle.psum(case.X, case.R1, case.R2[:, perm])
     np.testing.assert_allclose(b, a[perm], rtol=1e-13)
+
+
+# ------------------------------------------------------------------------------------------- shard merge
+def _shard_partials(case, bounds, k):
+    """Oracle routes of the expert ranges [bounds[s], bounds[s+1]) with ids made global; k_s = min(k, shard size)."""
+    S = len(bounds) - 1
+    T = case.X.shape[0]
+    idx = np.full((S, T, k), -1, dtype=np.int32)
+    val = np.full((S, T, k), -np.inf)
+    lse = np.zeros((S, T))
+    for s in range(S):
+        lo, hi = bounds[s], bounds[s + 1]
+        ks = min(k, hi - lo)
+        ref = oracle.route(case.X, case.R1, np.ascontiguousarray(case.R2[:, lo:hi]), ks, 1)
+        idx[s, :, :ks] = ref.idx + lo
+        val[s, :, :ks] = ref.topval
+        lse[s] = ref.lse
+    return idx, val, lse
+
+
+@pytest.mark.parametrize("gate_mode", [0, 1])
+@pytest.mark.parametrize("bounds", [(0, 96), (0, 48, 96), (0, 8, 40, 41, 96), (0, 3, 96)])
+def test_merge_of_expert_shards_equals_the_unsharded_route(bounds, gate_mode):
+    """A global top-k member is a top-k member of its own shard, and the shards' (m, Z) pairs combine like tiles in
+    Eq. app_online: merging the per-shard routes must reproduce the route over all experts (plain definition)."""
+    k = 6
+    case = inputs.gaussian_case(64, 32, 8, 96, k, gate_mode, seed=11)
+    full = oracle.route(case.X, case.R1, case.R2, k, gate_mode)
+    idx, val, lse = _shard_partials(case, bounds, k)
+    m_idx, m_gate, m_val, m_lse, m_counts = oracle.merge(idx, val, lse, 96, gate_mode)
+    assert np.array_equal(m_idx, full.idx)
+    np.testing.assert_allclose(m_val, full.topval, rtol=0, atol=0)          # the same fp64 numbers, only re-ordered
+    np.testing.assert_allclose(m_gate, full.gate, rtol=1e-12, atol=0)
+    np.testing.assert_allclose(m_lse, full.lse, rtol=1e-13, atol=1e-13)
+    assert np.array_equal(m_counts, full.counts)
+
+
+def test_merge_breaks_ties_by_ascending_id_and_ignores_unused_slots():
+    # two shards, one token, k = 3; equal logits 2.0 at ids 7 (shard 1) and 4 (shard 0): 4 goes first
+    idx = np.array([[[4, 1, -1]], [[7, 9, 8]]], dtype=np.int32)
+    val = np.array([[[2.0, 0.5, 123.0]], [[2.0, 3.0, -1.0]]])
+    m_idx, m_gate, m_val, m_lse, counts = oracle.merge(idx, val, None, 10, 0)
+    assert m_idx.tolist() == [[9, 4, 7]]
+    e = np.exp(np.array([3.0, 2.0, 2.0]) - 3.0)
+    np.testing.assert_allclose(m_gate[0], e / e.sum(), rtol=1e-15)
+    assert m_lse is None and counts.tolist() == [0, 0, 0, 0, 1, 0, 0, 1, 0, 1]
+    # fewer valid pairs than k: the tail is (-1, gate 0)
+    idx2 = np.array([[[5, -1, -1]]], dtype=np.int32)
+    val2 = np.array([[[1.0, 0.0, 0.0]]])
+    m_idx2, m_gate2, _, _, counts2 = oracle.merge(idx2, val2, None, 6, 0)
+    assert m_idx2.tolist() == [[5, -1, -1]] and m_gate2.tolist() == [[1.0, 0.0, 0.0]] and counts2.sum() == 1
+    with pytest.raises(ValueError):
+        oracle.merge(idx, val, None, 10, 1)                                  # full-softmax gates need the lse
