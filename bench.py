@@ -248,7 +248,8 @@ def unfused_reference_ms(torch, bufs, case, gate_mode, iters=5):
 
 def extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line):
     """Times the library's other entry points on the same inputs, each on its own (outside the router's timed region):
-    the dispatch bookkeeping that follows the router (Sort + Count) and Algorithm 2's second sweep (psum)."""
+    the dispatch bookkeeping that follows the router (Sort + Count), Algorithm 2's second sweep (psum) and the merge of
+    an expert-sharded router's reports."""
     X0, R10, R20, idx0, gate0, counts0 = bufs[0]
     mr.more_route(X0, R10, R20, k, gate_mode, idx0, gate0, counts0, stream)
     offs = torch.empty((case.M + 1,), dtype=torch.int32, device="cuda")
@@ -282,6 +283,28 @@ def extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line)
     rp = roofline(case.T, case.h, case.r, case.M, k, ps_secs, peaks)
     line["train_stats_psum"] = dict(us=ps_secs * 1e6, kernel="psum_tcgen05_kernel", bound=rp["bound"],
                                     roofline_frac=rp["frac"], psum_total=float(psum0.sum()), tokens=case.T)
+
+    # ---- the merge of an expert-sharded router: 8 shards' reports (here 8 copies of this router's own top-k with the
+    #      ids shifted, which is the same amount of work), timed on its own; HBM-bound: reads S*(8k+4) bytes per token
+    S = 8
+    tv0 = torch.empty((case.T, k), dtype=torch.float32, device="cuda")
+    mr.more_route_ex(X0, R10, R20, k, 1, idx0, gate0, counts0, tv0, lse0, 0, 0, stream)
+    sh_idx = (idx0.unsqueeze(0) // S).repeat(S, 1, 1).contiguous()
+    sh_val = tv0.unsqueeze(0).repeat(S, 1, 1).contiguous()
+    sh_lse = lse0.unsqueeze(0).repeat(S, 1).contiguous()
+    base = [s * (case.M // S) for s in range(S)]
+    for _ in range(3):
+        mr.more_merge_shards(sh_idx, sh_val, sh_lse, base, case.M, 1, idx0, gate0, counts0, None, None, stream)
+    d0.record(stream)
+    for _ in range(20):
+        mr.more_merge_shards(sh_idx, sh_val, sh_lse, base, case.M, 1, idx0, gate0, counts0, None, None, stream)
+    d1.record(stream)
+    stream.synchronize()
+    mg_us = d0.elapsed_time(d1) * 50.0
+    mg_bytes = case.T * (S * (8.0 * k + 4.0) + 8.0 * k)
+    line["merge_shards"] = dict(us=mg_us, shards=S, kernel="merge_shards_kernel",
+                                algorithmic_gbs=mg_bytes / (mg_us * 1e-6) / 1e9,
+                                hbm_frac=mg_bytes / (mg_us * 1e-6) / 1e9 / peaks["hbm_gbs"])
 
 
 

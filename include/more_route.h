@@ -154,6 +154,35 @@ int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h,
                     const float* lse, float* out_psum, int path, void* stream);
 
 /*
+ * more_merge_shards -- global top-k for a router whose EXPERT dimension is sharded (over GPUs, or over calls): the
+ * hierarchical top-k the paper's discussion of sharded routers leaves to future work ("each device computes a local
+ * top-k, then a global top-k"), with the shards' softmax statistics combined as in Eq. app_online.  Shard s has run
+ * more_route_ex on the same T tokens with its own slice R2[:, lo_s:hi_s] and reports out_idx, out_topval (and out_lse);
+ * after the reports of all S shards have been gathered into one buffer on this device (k pairs per token and shard),
+ * this call produces what an unsharded more_route would have: a global top-k member is always a top-k member of its
+ * own shard.
+ *
+ *   idx         device int32 [S][T][k]: expert ids as reported by the shards; shard_base[s] is added to those of shard s.
+ *               Slots with a negative id, with id + base >= M, or with a logit of -inf are unused (a shard with fewer
+ *               than k experts pads that way).
+ *   topval      device fp32 [S][T][k]: the logits of those ids (any order inside a row).
+ *   lse         device fp32 [S][T], or NULL: each shard's log-sum-exp over its own experts.  Required for
+ *               MORE_GATE_FULL_SOFTMAX; if given, out_lse = log sum_s exp(lse_s).
+ *   shard_base  HOST int32 [S], or NULL for all zeros (ids already global): first expert id of every shard.
+ *   S           1 .. MORE_MERGE_MAX_SHARDS;  k <= MORE_K_MAX.
+ *   out_idx, out_gate   device [T][k], as more_route: descending logit, ties by ascending global id; gates by gate_mode.
+ *               A token with fewer than k usable pairs gets id -1 and gate 0 in the remaining places.
+ *   out_topval  device fp32 [T][k] or NULL;  out_lse  device fp32 [T] or NULL.
+ *   out_counts  device int32 [M]: OVERWRITTEN with the histogram of out_idx.
+ * Asynchronous on `stream`; allocates nothing.  The selected logits are compared exactly as reported (no arithmetic
+ * on them before the comparison), so the result does not depend on how the experts were split.
+ */
+#define MORE_MERGE_MAX_SHARDS 64
+int more_merge_shards(const int32_t* idx, const float* topval, const float* lse, const int32_t* shard_base,
+                      int S, int T, int k, int M, int gate_mode, int32_t* out_idx, float* out_gate,
+                      float* out_topval, float* out_lse, int32_t* out_counts, void* stream);
+
+/*
  * more_dispatch -- dispatch bookkeeping for the grouped expert GEMMs that follow the router: the "Sort + Count" box
  * of the layer's forward flowchart ((N,k) -> (Nk) sorted indices + offsets).
  *

@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.more_route_psum.restype = i32
         L.more_dispatch.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.more_dispatch.restype = i32
+        L.more_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
+        L.more_merge_shards.restype = i32
         L.more_route_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
         L.more_route_noalloc.restype = i32
         L.more_route_noalloc_capacity.argtypes = []
@@ -175,6 +177,23 @@ def more_dispatch(idx, counts, out_offsets, out_sorted_pairs, stream=None):
     rc = lib().more_dispatch(_ptr(idx), _ptr(counts), T, k, M, _ptr(out_offsets), _ptr(out_sorted_pairs), _stream(stream))
     if rc != 0:
         raise MoreRouteError(rc, "more_dispatch")
+
+
+def more_merge_shards(idx, topval, lse, shard_base, M, gate_mode, out_idx, out_gate, out_counts, out_topval=None,
+                      out_lse=None, stream=None):
+    """``more_merge_shards`` of the C interface: ``idx``/``topval`` ``[S,T,k]`` (device), ``lse`` ``[S,T]`` or None,
+    ``shard_base`` a host sequence of S ints or None; fills ``out_idx``/``out_gate`` ``[T,k]`` and ``out_counts [M]``."""
+    S, T, k = idx.shape
+    base = None
+    if shard_base is not None:
+        base = (ctypes.c_int32 * S)(*[int(b) for b in shard_base])
+    rc = lib().more_merge_shards(_ptr(idx), _ptr(topval), _ptr(lse) if lse is not None else None,
+                                 ctypes.cast(base, ctypes.c_void_p) if base is not None else None,
+                                 S, T, k, M, gate_mode, _ptr(out_idx), _ptr(out_gate),
+                                 _ptr(out_topval) if out_topval is not None else None,
+                                 _ptr(out_lse) if out_lse is not None else None, _ptr(out_counts), _stream(stream))
+    if rc != 0:
+        raise MoreRouteError(rc, "more_merge_shards")
 
 
 def more_route_status(stream=None) -> int:
