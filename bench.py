@@ -302,6 +302,22 @@ def extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line)
     stream.synchronize()
     mg_us = d0.elapsed_time(d1) * 50.0
     mg_bytes = case.T * (S * (8.0 * k + 4.0) + 8.0 * k)
+    # ---- the fused standard (full-rank) router on the same (T, h, M, k): a T x h x M contraction with the same
+    #      selection epilogue (the paper's "fused standard MoE" comparison); W is random, timed on its own
+    Wf = (torch.randn((case.h, case.M), device="cuda") / case.h ** 0.5).to(torch.bfloat16)
+    for _ in range(2):
+        mr.more_route_full(X0, Wf, k, gate_mode, idx0, gate0, counts0, None, None, 0, stream)
+    d0.record(stream)
+    for _ in range(5):
+        mr.more_route_full(X0, Wf, k, gate_mode, idx0, gate0, counts0, None, None, 0, stream)
+    d1.record(stream)
+    stream.synchronize()
+    fr_secs = d0.elapsed_time(d1) * 1e-3 / 5
+    fr_tflops = 2.0 * case.T * case.h * case.M / fr_secs / 1e12
+    line["standard_router_fused"] = dict(us=fr_secs * 1e6, kernel="route_tcgen05_kernel<.., FULL>", tflops=fr_tflops,
+                                         tensor_frac=fr_tflops / peaks["bf16_tflops_sustained"],
+                                         peak="measured bf16 (sustained: the kernel runs for milliseconds)")
+    del Wf
     line["merge_shards"] = dict(us=mg_us, shards=S, kernel="merge_shards_kernel",
                                 algorithmic_gbs=mg_bytes / (mg_us * 1e-6) / 1e9,
                                 hbm_frac=mg_bytes / (mg_us * 1e-6) / 1e9 / peaks["hbm_gbs"])

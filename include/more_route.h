@@ -154,6 +154,23 @@ int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h,
                     const float* lse, float* out_psum, int path, void* stream);
 
 /*
+ * more_route_full -- the fused STANDARD (full-rank) router, g(x) = softmax(TopK(R x)): the same sweep without the
+ * low-rank bottleneck (Algorithm 1 with the contraction running over K = h instead of r; the paper's "fused standard
+ * MoE" comparison).  Logits l = X W with W = R^T stored [h][M] row-major; they are produced 64 experts at a time by
+ * accumulating over all of h on the tensor cores, and selected, gated and counted exactly as in more_route.  The
+ * T x M logits never reach memory, but X is re-read (from L2) once per 64-expert step, so unlike the low-rank router
+ * this one does a full T x h x M contraction.
+ *
+ *   X           device bf16 [T][h];  W  device bf16 [h][M];  both 16-byte aligned; h and M multiples of 8, k <= 32
+ *               (other shapes: MORE_ERR_SHAPE -- this entry point has the tensor-core path only).
+ *   gate_mode, out_idx, out_gate, out_counts, out_topval, out_lse, msplit, stream: as for more_route_ex.
+ * The products of bf16 inputs are exact in fp32 and only the fp32 accumulation rounds, so the logits agree with exact
+ * arithmetic to ~1e-6 relative.
+ */
+int more_route_full(const void* X, const void* W, int T, int h, int M, int k, int gate_mode, int32_t* out_idx,
+                    float* out_gate, int32_t* out_counts, float* out_topval, float* out_lse, int msplit, void* stream);
+
+/*
  * more_merge_shards -- global top-k for a router whose EXPERT dimension is sharded (over GPUs, or over calls): the
  * hierarchical top-k the paper's discussion of sharded routers leaves to future work ("each device computes a local
  * top-k, then a global top-k"), with the shards' softmax statistics combined as in Eq. app_online.  Shard s has run

@@ -48,6 +48,8 @@ def lib() -> ctypes.CDLL:
         L.more_route_psum.restype = i32
         L.more_dispatch.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
         L.more_dispatch.restype = i32
+        L.more_route_full.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, vp]
+        L.more_route_full.restype = i32
         L.more_merge_shards.argtypes = [vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp]
         L.more_merge_shards.restype = i32
         L.more_route_noalloc.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, vp, vp, vp]
@@ -177,6 +179,17 @@ def more_dispatch(idx, counts, out_offsets, out_sorted_pairs, stream=None):
     rc = lib().more_dispatch(_ptr(idx), _ptr(counts), T, k, M, _ptr(out_offsets), _ptr(out_sorted_pairs), _stream(stream))
     if rc != 0:
         raise MoreRouteError(rc, "more_dispatch")
+
+
+def more_route_full(X, W, k, gate_mode, out_idx, out_gate, out_counts, out_topval=None, out_lse=None, msplit=0,
+                    stream=None):
+    """``more_route_full`` of the C interface: the fused standard router, logits ``X [T,h] @ W [h,M]`` (bf16, device)."""
+    T, h = X.shape
+    M = W.shape[1]
+    rc = lib().more_route_full(_ptr(X), _ptr(W), T, h, M, k, gate_mode, _ptr(out_idx), _ptr(out_gate), _ptr(out_counts),
+                               _ptr(out_topval), _ptr(out_lse), msplit, _stream(stream))
+    if rc != 0:
+        raise MoreRouteError(rc, "more_route_full")
 
 
 def more_merge_shards(idx, topval, lse, shard_base, M, gate_mode, out_idx, out_gate, out_counts, out_topval=None,

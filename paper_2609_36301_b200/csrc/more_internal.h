@@ -20,6 +20,7 @@ struct RouteArgs {
     float* out_topval;  // nullable
     float* out_lse;     // nullable
     cudaStream_t stream;
+    bool full = false;  // standard (full-rank) router: R1 unused, R2 is W [h][M], r only sizes the plan
 };
 
 // Per-device state: one cached scratch allocation, the sticky status word, device facts.

@@ -68,7 +68,7 @@ int route_device(const RouteArgs& a, int path, int msplit)
     int rc = check_shape(a.T, a.h, a.r, a.M, a.k, a.gate_mode, path);
     if (rc != MORE_OK) return rc;
     if (!a.out_counts) return MORE_ERR_NULL;
-    if (a.T > 0 && (!a.X || !a.R1 || !a.R2 || !a.out_idx || !a.out_gate)) return MORE_ERR_NULL;
+    if (a.T > 0 && (!a.X || (!a.R1 && !a.full) || !a.R2 || !a.out_idx || !a.out_gate)) return MORE_ERR_NULL;
     if (!aligned(a.X, 16) || !aligned(a.R1, 16) || !aligned(a.R2, 16)) return MORE_ERR_ALIGN;
     if (!aligned(a.out_idx, 4) || !aligned(a.out_gate, 4) || !aligned(a.out_counts, 4) || !aligned(a.out_topval, 4) ||
         !aligned(a.out_lse, 4))
@@ -165,6 +165,23 @@ int more_route_ex(const void* X, const void* R1, const void* R2, int T, int h, i
     a.out_topval = out_topval; a.out_lse = out_lse;
     a.stream = static_cast<cudaStream_t>(stream);
     return route_device(a, path, msplit);
+}
+
+int more_route_full(const void* X, const void* W, int T, int h, int M, int k, int gate_mode, int32_t* out_idx,
+                    float* out_gate, int32_t* out_counts, float* out_topval, float* out_lse, int msplit, void* stream)
+{
+    // the standard router has only the tensor-core path: say so instead of silently doing something else
+    if (h < 1 || M < 1 || h % 8 != 0 || M % 8 != 0) return MORE_ERR_SHAPE;
+    RouteArgs a;
+    a.X = static_cast<const __nv_bfloat16*>(X);
+    a.R1 = nullptr;
+    a.R2 = static_cast<const __nv_bfloat16*>(W);
+    a.T = T; a.h = h; a.r = 64; a.M = M; a.k = k; a.gate_mode = gate_mode;   // r: the plan's cost model only
+    a.out_idx = out_idx; a.out_gate = out_gate; a.out_counts = out_counts;
+    a.out_topval = out_topval; a.out_lse = out_lse;
+    a.stream = static_cast<cudaStream_t>(stream);
+    a.full = true;
+    return route_device(a, MORE_PATH_TCGEN05, msplit);
 }
 
 int more_route(const void* X, const void* R1, const void* R2, int T, int h, int r, int M, int k, int gate_mode,

@@ -100,14 +100,12 @@ constexpr int kCandColStride = kEpilogueThreads * 4;      // ... and between its
 #ifndef MORE_CAND_CAP
 #define MORE_CAND_CAP 12
 #endif
-#ifndef MORE_WARN
-#define MORE_WARN (MORE_CAND_CAP - 4)
-#endif
-static_assert(MORE_WARN >= 1 && MORE_WARN <= MORE_CAND_CAP - 4, "a chunk must always find 4 free slots");
 constexpr unsigned kFullMask = 0xffffffffu;
 
 template <int KCAP, int CAP>
 struct Selector {
+    static constexpr int kWarnSlots = CAP - 4;            // a chunk must always find 4 free slots
+    static_assert(kWarnSlots >= 1, "candidate buffer too small");
     TopList<KCAP> L;
     float tau;
     uint32_t ptr;     // shared-memory address of this thread's next free value slot
@@ -121,7 +119,7 @@ struct Selector {
         tau = -INFINITY;
         base = ptr = first_val_slot;
         cbase = cptr = first_col_slot;
-        warn = first_val_slot + MORE_WARN * kCandValStride;
+        warn = first_val_slot + kWarnSlots * kCandValStride;
     }
     // Called by all 32 lanes of a warp together.  Every round inserts at most one element per token: the maximum
     // of the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
@@ -227,7 +225,11 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
 }
 
 // ------------------------------------------------------------------------------------------------- the kernel
-template <int RPAD, int KCAP, bool LSE>
+// FULL = true is the fused STANDARD router (logits = X W with W [h][M], no low-rank bottleneck: Alg. 1 without z, the
+// contraction running over K = h): there is no phase 1, every 64-expert step instead accumulates over all h/64 k-tiles
+// of X (256 x 64, re-read per step) and W (64 x 64) with the phase-1 pipeline and stage layout, and the epilogue is
+// the same.  map_r2 is then W's map (64 x 64 boxes), map_r1 is unused, RPAD is 64.
+template <int RPAD, int KCAP, bool LSE, bool FULL = false>
 __global__ void __launch_bounds__(kThreads, 2)
 route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
                      const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
@@ -235,11 +237,14 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
     constexpr int kHalf = 64;                                   // experts per phase-2 step: one 128-byte-wide R2 block
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
-    constexpr int kStagesP2 = (RPAD == 64) ? 6 : 8;             // R2 blocks in flight
-    constexpr int kCandCap = MORE_CAND_CAP;                     // candidate slots per token
+    constexpr int kStagesP2 = FULL ? 1 : ((RPAD == 64) ? 6 : 8);   // R2 blocks in flight (unused by FULL)
+    // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
+    constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
+    using Sel = Selector<KCAP, kCandCap>;
     constexpr int kCandValBytes = kCandCap * kCandValStride;
     constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);
-    static_assert(kCandBytes + kStagesP2 * kR2StageBytes <= kRingBytes, "phase-2 layout does not fit");
+    constexpr int kCandOffset = FULL ? kStagesP1 * kP1StageBytes : 0;
+    static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRingBytes, "phase-2 layout does not fit");
     // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
     // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.
     constexpr uint32_t kAccCols = 64, kZopCol0 = 128;
@@ -290,7 +295,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t cand = ring;                                 // phase 2: candidate buffers
+    const uint32_t cand = ring + kCandOffset;                   // phase 2: candidate buffers
     const uint32_t r2ring = ring + kCandBytes;                  // phase 2: R2 stages
     // 64-expert steps of this CTA (the last one of the last tile is skipped when it lies wholly beyond M)
     const int e_lo = tile_lo * kTileExperts;
@@ -299,7 +304,20 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
-        if (lane == 0) {
+        if (lane == 0 && FULL) {
+            // standard router: for every 64-expert step, all k-tiles of X and of W[:, step]
+            bool ok = true;
+            const int total = nsteps * ktiles1;
+            for (int g = 0; g < total && ok; ++g) {
+                const int s = g % kStagesP1, it = g / ktiles1, kt = g % ktiles1;
+                if (g >= kStagesP1) ok = mbar_wait(bar(B_EMPTY1 + s), ((g / kStagesP1) - 1) & 1, abort_flag, p.status);
+                if (!ok) break;
+                const uint32_t dst = ring + s * kP1StageBytes;
+                mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
+                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // 256 token rows x 64 columns
+                tma_load_2d(dst + kXTileBytes, &map_r2, bar(B_FULL1 + s), e_lo + it * kHalf, kt * 64);
+            }
+        } else if (lane == 0) {
             bool ok = true;
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
                 const int s = kt % kStagesP1;
@@ -326,6 +344,40 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         bool ok = true;
         constexpr uint32_t idesc1 = umma_idesc(64);
         constexpr uint32_t idesc2 = umma_idesc(kHalf);
+        if constexpr (FULL) {
+            // standard router: per 64-expert step, K runs over all of h through the two k-tile stages
+            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), wd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
+            const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), w_lo0 = (uint32_t)wd, w_hi = (uint32_t)(wd >> 32);
+            int g = 0;
+            for (int it = 0; it < nsteps && ok; ++it) {
+                // both accumulators must have been read out (the k-tiles serve both token groups)
+#pragma unroll
+                for (int a = 0; a < 2; ++a)
+                    if (a * 128 < p.block_tokens)
+                        ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
+                if (!ok) break;
+                for (int kt = 0; kt < ktiles1 && ok; ++kt, ++g) {
+                    const int s = g % kStagesP1;
+                    ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (g / kStagesP1) & 1, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), w_lo = w_lo0 + s * (kP1StageBytes >> 4);
+#pragma unroll
+                    for (int a = 0; a < 2; ++a) {
+                        if (a * 128 >= p.block_tokens) continue;
+#pragma unroll
+                        for (int kk = 0; kk < 4; ++kk)
+                            tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
+                                                 w_lo + kk * (2048 >> 4), w_hi, idesc1, (kt | kk) != 0);
+                    }
+                    tc_commit_elect(bar(B_EMPTY1 + s));
+                }
+                if (!ok) break;
+#pragma unroll
+                for (int a = 0; a < 2; ++a)
+                    if (a * 128 < p.block_tokens) tc_commit_elect(bar(B_ACCF + a));
+            }
+        } else {
         {
             // descriptor words of stage 0: K-major X tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address
             const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
@@ -372,6 +424,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             if (!ok) break;
             tc_commit_elect(bar(B_EMPTY2 + s));
         }
+        }   // !FULL
     } else {
         // ========================================================================================= epilogue
         const int q = warp & 3;                              // TMEM lane group this warp may read
@@ -384,9 +437,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
         const uint32_t t_zop = tmem_base + ((uint32_t)(q * 32) << 16) + kZopCol0 + acc * 64;
         STAT(const long long st_k0 = clock64();)
-        bool ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
+        bool ok = FULL ? true : mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
         STAT(const long long st_k1 = clock64();)
-        if (ok) {
+        if (ok && !FULL) {
             // ---- narrow z to bf16 [hi | lo] and store it to tensor memory as the A operand of phase 2
             tc_fence_after();
 #pragma unroll
@@ -411,7 +464,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             mbar_arrive(bar(B_ZOP));
         }
 
-        Selector<KCAP, kCandCap> S;
+        Sel S;
         S.init(cand + row_in_blk * 16, cand + kCandValBytes + row_in_blk * 4);
         STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_rcall = 0, st_riter = 0; long long st_twait = 0, st_tproc = 0, st_tref = 0;
              const long long st_t0 = clock64();)
@@ -464,7 +517,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     S.scan(v, t, col0);
                     STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
                     const uint32_t fill = __reduce_max_sync(kFullMask, S.ptr - S.base);
-                    if (fill >= MORE_WARN * kCandValStride) {
+                    if (fill >= Sel::kWarnSlots * kCandValStride) {
                         // some token is about to run out of slots: fold now
                         STAT(st_rcall++; st_riter += fill / kCandValStride; const long long tr0 = clock64();)
                         S.refresh();
@@ -670,12 +723,12 @@ int get_tensor_map(const void* ptr, int rows, int cols, int box_rows, int box_co
 
 namespace {
 
-template <int RPAD, int KCAP, bool LSE>
+template <int RPAD, int KCAP, bool LSE, bool FULL>
 int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp, int ctas,
                cudaStream_t st)
 {
     static unsigned long long configured = 0;   // one bit per device, per instantiation; guarded by the API mutex
-    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE>;
+    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE, FULL>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (!(configured >> (dev & 63) & 1ull)) {
@@ -688,24 +741,24 @@ int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& 
     return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
 }
 
-template <int RPAD, int KCAP>
+template <int RPAD, int KCAP, bool FULL>
 int launch_lse(bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp,
                int ctas, cudaStream_t st)
 {
-    return lse ? launch_one<RPAD, KCAP, true>(mx, m1, m2, kp, ctas, st)
-               : launch_one<RPAD, KCAP, false>(mx, m1, m2, kp, ctas, st);
+    return lse ? launch_one<RPAD, KCAP, true, FULL>(mx, m1, m2, kp, ctas, st)
+               : launch_one<RPAD, KCAP, false, FULL>(mx, m1, m2, kp, ctas, st);
 }
 
-template <int RPAD>
+template <int RPAD, bool FULL = false>
 int launch_kcap(int k, bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2,
                 const KernelParams& kp, int ctas, cudaStream_t st)
 {
-    if (k <= 8) return launch_lse<RPAD, 8>(lse, mx, m1, m2, kp, ctas, st);
+    if (k <= 8) return launch_lse<RPAD, 8, FULL>(lse, mx, m1, m2, kp, ctas, st);
 #ifdef MORE_ONLY_K8
     return MORE_ERR_SHAPE;
 #endif
-    if (k <= 16) return launch_lse<RPAD, 16>(lse, mx, m1, m2, kp, ctas, st);
-    return launch_lse<RPAD, 32>(lse, mx, m1, m2, kp, ctas, st);
+    if (k <= 16) return launch_lse<RPAD, 16, FULL>(lse, mx, m1, m2, kp, ctas, st);
+    return launch_lse<RPAD, 32, FULL>(lse, mx, m1, m2, kp, ctas, st);
 }
 
 int kcap_of(int k) { return k <= 8 ? 8 : (k <= 16 ? 16 : 32); }
@@ -731,9 +784,15 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
 {
     CUtensorMap mx, m1, m2;
     int rc = get_tensor_map(a.X, a.T, a.h, kBlockTokens, 64, &mx);
-    if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
-    const int rpad = (a.r <= 16) ? 16 : (a.r <= 32 ? 32 : 64);
-    if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.r, a.M, rpad, 64, &m2);
+    const int rpad = a.full ? 64 : ((a.r <= 16) ? 16 : (a.r <= 32 ? 32 : 64));
+    if (a.full) {
+        // standard router: R2 is W [h][M]; its k-tiles are 64 x 64 boxes like R1's
+        if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.h, a.M, 64, 64, &m2);
+        m1 = m2;
+    } else {
+        if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
+        if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.r, a.M, rpad, 64, &m2);
+    }
     if (rc != MORE_OK) return rc;
 
     KernelParams kp;
@@ -760,6 +819,7 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
         if (cudaMemsetAsync(kp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
     }
     const bool lse = (a.gate_mode == MORE_GATE_FULL_SOFTMAX) || (a.out_lse != nullptr);
+    if (a.full) return launch_kcap<64, true>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
     switch (rpad) {
         case 16: return launch_kcap<16>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
         case 32: return launch_kcap<32>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
