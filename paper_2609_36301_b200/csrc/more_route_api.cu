@@ -117,7 +117,8 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
     // Fill one wave of resident CTAs as evenly as possible.  Candidates: tokens per CTA (a multiple of 32 up to
     // 256; smaller blocks waste rows of the second accumulator but even out the SMs) x CTAs per token block
     // (each extra CTA repeats the block's z projection and starts its top-k from scratch, and a second, partial
-    // wave costs more than it gains; every CTA keeps at least four expert tiles).
+    // wave costs more than it gains; every CTA keeps at least twelve expert tiles -- the first few hundred experts
+    // of a sweep cost far more than the rest, so short sweeps are not worth starting twice).
     double best = 1e300;
     int best_bt = kBlockTokens, best_s = 1;
     for (int bt = kBlockTokens; bt >= 128; bt -= 32) {
@@ -125,7 +126,7 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
         int s = msplit;
         if (s == 0) {
             s = slots / blocks;
-            if (s > tiles / 4) s = tiles / 4;
+            if (s > tiles / 12) s = tiles / 12;
             if (s < 1) s = 1;
             if (s > 64) s = 64;
         }
