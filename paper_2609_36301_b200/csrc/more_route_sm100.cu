@@ -98,7 +98,7 @@ struct TopList {
 constexpr int kCandValStride = kEpilogueThreads * 16;     // bytes between successive value slots of one thread
 constexpr int kCandColStride = kEpilogueThreads * 4;      // ... and between its column slots
 #ifndef MORE_CAND_CAP
-#define MORE_CAND_CAP 12
+#define MORE_CAND_CAP 8
 #endif
 constexpr unsigned kFullMask = 0xffffffffu;
 
@@ -237,12 +237,15 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
     constexpr int kHalf = 64;                                   // experts per phase-2 step: one 128-byte-wide R2 block
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
-    constexpr int kStagesP2 = FULL ? 1 : ((RPAD == 64) ? 6 : 8);   // R2 blocks in flight (unused by FULL)
     // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
     constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
     using Sel = Selector<KCAP, kCandCap>;
     constexpr int kCandValBytes = kCandCap * kCandValStride;
     constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);
+    // R2 blocks in flight: what the ring has room for next to the candidate buffers, at most 8 (unused by FULL)
+    constexpr int kStagesFit = (kRingBytes - kCandBytes) / kR2StageBytes;
+    constexpr int kStagesP2 = FULL ? 1 : (kStagesFit < 8 ? kStagesFit : 8);
+    static_assert(FULL || kStagesP2 >= 2, "no room for the R2 pipeline");
     constexpr int kCandOffset = FULL ? kStagesP1 * kP1StageBytes : 0;
     static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRingBytes, "phase-2 layout does not fit");
     // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
