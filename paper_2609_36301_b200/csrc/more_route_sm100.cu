@@ -519,10 +519,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     STAT(st_hit++; const uint32_t mark = S.ptr;)
                     S.scan(v, t, col0);
                     STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
-                    const uint32_t fill = __reduce_max_sync(kFullMask, S.ptr - S.base);
-                    if (fill >= Sel::kWarnSlots * kCandValStride) {
+                    if (__any_sync(kFullMask, S.ptr >= S.warn)) {
                         // some token is about to run out of slots: fold now
-                        STAT(st_rcall++; st_riter += fill / kCandValStride; const long long tr0 = clock64();)
+                        STAT(st_rcall++; const long long tr0 = clock64();)
                         S.refresh();
                         STAT(st_tref += clock64() - tr0;)
                     }
