@@ -117,7 +117,7 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
     // Fill one wave of resident CTAs as evenly as possible.  Candidates: tokens per CTA (a multiple of 32 up to
     // 256; smaller blocks waste rows of the second accumulator but even out the SMs) x CTAs per token block
     // (each extra CTA repeats the block's z projection and starts its top-k from scratch, and a second, partial
-    // wave costs more than it gains; every CTA keeps at least twelve expert tiles -- the first few hundred experts
+    // wave costs more than it gains; every CTA keeps at least eight expert tiles -- the first few hundred experts
     // of a sweep cost far more than the rest, so short sweeps are not worth starting twice).
     double best = 1e300;
     int best_bt = kBlockTokens, best_s = 1;
@@ -125,8 +125,16 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
         const int blocks = (T + bt - 1) / bt;
         int s = msplit;
         if (s == 0) {
+            // while the CTAs have an SM each, splitting is cheap: keep eight tiles per CTA; once two CTAs share an
+            // SM the second one gains less than its repeated start costs: keep sixteen
             s = slots / blocks;
-            if (s > tiles / 12) s = tiles / 12;
+            if (s > tiles / 8) s = tiles / 8;
+            if ((long long)blocks * s > sm_count) {
+                int dense = s < tiles / 16 ? s : tiles / 16;
+                const int one_per_sm = sm_count / blocks;
+                s = dense > one_per_sm ? dense : one_per_sm;
+                if (s > tiles / 8) s = tiles / 8;
+            }
             if (s < 1) s = 1;
             if (s > 64) s = 64;
         }

@@ -625,11 +625,35 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     TopList<KCAP> G;
                     G.init();
                     float gm = -INFINITY, gz = 0.f;
+                    // A token's partial lists lie one after the other in scratch.  Each list's head (its four best
+                    // entries, which is all most lists contribute) is fetched with two 16-byte loads, and the next
+                    // list's head is requested before the current one is merged, so the L2 round trips overlap
+                    // instead of adding up; the tail of a list is read only if its fourth entry still got in.
+                    const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
+                    const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
+                    float4 hv = __ldcg(pv);
+                    int4 hi = __ldcg(pi);
                     for (int sp = 0; sp < p.msplit; ++sp) {       // ascending expert ranges: ties keep the smaller id
-                        for (int s = 0; s < KCAP; ++s) {
+                        const float4 cv = hv;
+                        const int4 ci = hi;
+                        if (sp + 1 < p.msplit) {
+                            hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
+                            hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
+                        }
+                        // each partial list is sorted: stop at the first entry that does not get in
+                        bool more = cv.x > G.tau();
+                        if (more) G.insert(cv.x, ci.x);
+                        more = more && cv.y > G.tau();
+                        if (more) G.insert(cv.y, ci.y);
+                        more = more && cv.z > G.tau();
+                        if (more) G.insert(cv.z, ci.z);
+                        more = more && cv.w > G.tau();
+                        if (more) G.insert(cv.w, ci.w);
+                        for (int s = 4; s < KCAP && more; ++s) {
                             const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
                             const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
-                            if (x > G.tau()) G.insert(x, j); else break;   // each partial list is sorted
+                            more = x > G.tau();
+                            if (more) G.insert(x, j);
                         }
                         const float2 mz = __ldcg(p.part_mz + base + sp);
                         if (LSE && mz.x > -INFINITY) {
