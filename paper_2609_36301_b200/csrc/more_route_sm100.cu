@@ -178,7 +178,8 @@ struct Selector {
 
 struct KernelParams {
     int T, h, r, M, k, gate_mode, msplit;
-    int block_tokens;            // tokens routed per CTA: a multiple of 32, at most 256 (the X tile always has 256 rows)
+    int block_tokens;            // tokens routed per CTA: a multiple of 32, at most 256
+    int x_rows;                  // rows of the X tile: 256, or 128 when block_tokens <= 128 (low-rank router only)
     int tiles_total;             // ceil(M / 128)
     int32_t* out_idx;
     float* out_gate;
@@ -260,7 +261,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint8_t* ctl = ring_ptr + kRingBytes;                    // control block
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
     // barrier slots
-    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kStagesP1, B_ZACC = B_EMPTY1 + kStagesP1, B_ZOP = B_ZACC + 1,
+    constexpr int kMaxStagesP1 = 4;
+    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kMaxStagesP1, B_ZACC = B_EMPTY1 + kMaxStagesP1, B_ZOP = B_ZACC + 1,
                   B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
                   B_COUNT = B_ACCE + 2;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
@@ -277,9 +279,14 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int tile_lo = (int)(((long long)p.tiles_total * split) / p.msplit);
     const int tile_hi = (int)(((long long)p.tiles_total * (split + 1)) / p.msplit);
     const int ktiles1 = (p.h + 63) / 64;
+    // phase-1 stages: a 128-row X tile (small token blocks) leaves room for four k-tiles in flight instead of two,
+    // which matters when a CTA's projection is a chain of L2 round trips rather than a stream
+    const int x_tile_bytes = p.x_rows * 128;
+    const int st1_bytes = x_tile_bytes + kR1TileBytes;
+    const int nst1 = (p.x_rows == 128) ? 4 : kStagesP1;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kStagesP1; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
+        for (int i = 0; i < kMaxStagesP1; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
         mbar_init(bar(B_ZACC), 1);
         mbar_init(bar(B_ZOP), kEpilogueThreads);
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
@@ -323,13 +330,13 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         } else if (lane == 0) {
             bool ok = true;
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
-                const int s = kt % kStagesP1;
-                if (kt >= kStagesP1) ok = mbar_wait(bar(B_EMPTY1 + s), ((kt / kStagesP1) - 1) & 1, abort_flag, p.status);
+                const int s = kt % nst1;
+                if (kt >= nst1) ok = mbar_wait(bar(B_EMPTY1 + s), ((kt / nst1) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t dst = ring + s * kP1StageBytes;
-                mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
-                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // 256 token rows x 64 columns
-                tma_load_2d(dst + kXTileBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
+                const uint32_t dst = ring + s * st1_bytes;
+                mbar_expect_tx(bar(B_FULL1 + s), st1_bytes);
+                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // x_rows token rows x 64 columns
+                tma_load_2d(dst + x_tile_bytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
             }
             // the ring is reused by phase 2: wait until every phase-1 MMA has finished reading it
             ok = ok && mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
@@ -383,16 +390,17 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         } else {
         {
             // descriptor words of stage 0: K-major X tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address
-            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
+            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + x_tile_bytes, 8192, 1024);
             const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
-                const int s = kt % kStagesP1;
-                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / kStagesP1) & 1, abort_flag, p.status));
+                const int s = kt % nst1;
+                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / nst1) & 1, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), r_lo = r_lo0 + s * (kP1StageBytes >> 4);
+                const uint32_t x_lo = x_lo0 + s * (st1_bytes >> 4), r_lo = r_lo0 + s * (st1_bytes >> 4);
 #pragma unroll
                 for (int a = 0; a < 2; ++a) {
+                    if (a * 128 >= p.x_rows) continue;      // a 128-row X tile has no second token group
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
                         tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
@@ -809,7 +817,8 @@ size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p)
 int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
 {
     CUtensorMap mx, m1, m2;
-    int rc = get_tensor_map(a.X, a.T, a.h, kBlockTokens, 64, &mx);
+    const int x_rows = (!a.full && p.block_tokens <= 128) ? 128 : kBlockTokens;
+    int rc = get_tensor_map(a.X, a.T, a.h, x_rows, 64, &mx);
     const int rpad = a.full ? 64 : ((a.r <= 16) ? 16 : (a.r <= 32 ? 32 : 64));
     if (a.full) {
         // standard router: R2 is W [h][M]; its k-tiles are 64 x 64 boxes like R1's
@@ -824,6 +833,7 @@ int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     KernelParams kp;
     kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
     kp.block_tokens = p.block_tokens;
+    kp.x_rows = x_rows;
     kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
     kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
     kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
