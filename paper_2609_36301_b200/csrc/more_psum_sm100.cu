@@ -229,7 +229,9 @@ psum_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     acc0 += ex2f(fmaf(v[4 * g], kLog2e, -l.x));
                     acc1 += ex2f(fmaf(v[4 * g + 1], kLog2e, -l.y));
                     acc2 += ex2f(fmaf(v[4 * g + 2], kLog2e, -l.z));
-                    acc3 += ex2f(fmaf(v[4 * g + 3], kLog2e, -l.w));
+                    // (one exponential in four on the FMA pipe: the special-function unit's 16 results per clock per SM
+                    // are this loop's narrowest resource; more than one in four costs more issue slots than it frees)
+                    acc3 += ex2_poly(fmaf(v[4 * g + 3], kLog2e, -l.w));
                 }
             };
             tmem_ld16(t_lane, va);

@@ -150,6 +150,22 @@ __device__ __forceinline__ void tc_commit_elect(uint32_t bar)
         "@pe tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}" ::"r"(bar) : "memory");
 }
 
+// 2^x for x <= 0 without the special-function unit: x = n + f with n = round(x) (the 1.5 * 2^23 trick leaves n in
+// the low mantissa bits of t), 2^f by a degree-4 polynomial on [-0.5, 0.5] (relative error < 5e-5), and the exponent
+// added as an integer.  Seven of its nine instructions run on the FMA pipe.
+__device__ __forceinline__ float ex2_poly(float x)
+{
+    x = fmaxf(x, -125.f);
+    const float t = x + 12582912.f;
+    const float f = x - (t - 12582912.f);
+    float p = 0.00961813f;
+    p = fmaf(p, f, 0.0555041f);
+    p = fmaf(p, f, 0.240227f);
+    p = fmaf(p, f, 0.693147f);
+    p = fmaf(p, f, 1.0f);
+    return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
+
 // Store 8 consecutive 32-bit columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&u)[8])
 {
