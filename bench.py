@@ -69,7 +69,7 @@ def roofline(T, h, r, M, k, seconds, peaks, traffic=None):
 # DRAM bytes per launch of route_tcgen05_kernel from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum);
 # the capture behind each figure is summarised under profiles/.  None = not captured for that workload.
 NCU_TRAFFIC_BYTES = {
-    "c3": 275.2e6,          # profiles/route_tcgen05_kernel_c3_ncu_full.md
+    "c3": 274.5e6,          # profiles/route_tcgen05_kernel_c3_ncu_full.md
     "c2_M16384": 34.78e6,   # profiles/route_tcgen05_kernel_c2_M16384_ncu_full.md
 }
 
