@@ -5,8 +5,9 @@
 // One CTA routes one block of 256 tokens (two 128-row accumulators) over one contiguous range of expert tiles
 // (Algorithm 1, with the token block additionally split over `msplit` CTAs along the expert dimension):
 //
-//   phase 1  z = X_blk R1            TMA streams 256x64 X tiles and 64x64 R1 tiles (zero-filled beyond r),
-//                                    tcgen05.mma accumulates two 128 x 64 fp32 blocks in TMEM.
+//   phase 1  z = X_blk R1            TMA streams 256x64 X tiles (128x64 and twice the stages for blocks of at most 128
+//                                    tokens) and 64x64 R1 tiles (zero-filled beyond r), tcgen05.mma accumulates two
+//                                    128 x 64 fp32 blocks in TMEM.
 //   narrow   z -> bf16 hi + bf16 lo  written back to tensor memory (tcgen05.st) as the A operands [hi | lo] of phase 2:
 //                                    TMEM lane = token, two K-elements per 32-bit column.  Carrying both parts keeps
 //                                    the logits within ~3e-5 of exact arithmetic.
@@ -24,8 +25,8 @@
 // Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue (the whole warp stays converged and one
 // elected lane issues; see tc_mma_bf16_ts_elect), warps 2..9 = epilogue (warp w reads TMEM lanes 32*(w%4).. of
 // accumulator (w-2)/4).  Two CTAs are resident per SM (256 TMEM columns and ~112 KB of shared memory each): while one
-// group's epilogue drains its accumulator the MMAs of the other three groups of the SM run, and one CTA's HBM-bound
-// phase 1 overlaps the other's expert sweep.
+// group's epilogue drains its accumulator the MMAs of the other three groups of the SM run.  The same kernel with
+// FULL = true is the fused standard router (no z; every step contracts over all of h).
 //
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
 // status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
@@ -489,7 +490,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             const int e0 = e_lo + it * kHalf;
             const bool ragged = e0 + kHalf > p.M;
             float va[16], vb[16];
-            // ---- one 16-column chunk: triple maxima, optional online softmax update, candidate scan
+            // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate scan
             auto process = [&](float (&v)[16], int col0) {
 #ifdef MORE_EXP_NOPROC
                 return;
