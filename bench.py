@@ -467,6 +467,10 @@ def main():
                 others[f"{oname}/mode{gm}"] = dict(us=osecs * 1e6, tokens_per_s=ocase.T / osecs, bound=r["bound"],
                                                     roofline_frac=r["frac"],
                                                     msplit=mr.more_route_plan(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k).msplit)
+                if oname.startswith("c2_") and not args.no_context:
+                    # the expert-count sweep's fused vs unfused-logits comparison (library ops, logits in HBM)
+                    ums = unfused_reference_ms(torch, obufs, ocase, gm, iters=3)
+                    others[f"{oname}/mode{gm}"]["unfused_gpu_reference_us"] = None if ums is None else ums * 1e3
                 del obufs
             torch.cuda.empty_cache()
         line["others"] = others
