@@ -59,6 +59,8 @@ def lib() -> ctypes.CDLL:
         ip = ctypes.POINTER(ctypes.c_int)
         L.more_route_plan.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, ip, ip, ip]
         L.more_route_plan.restype = i32
+        L.more_route_plan_ex.argtypes = [i32, i32, i32, i32, i32, i32, i32, i32, i32, ip]
+        L.more_route_plan_ex.restype = i32
         L.more_route_status.argtypes = [vp]
         L.more_route_status.restype = i32
         L.more_route_launches.argtypes = []
@@ -88,6 +90,10 @@ class RoutePlan:
     path: int
     msplit: int
     ctas: int
+    block_tokens: int = 0
+    token_groups: int = 1
+    expert_ranges: int = 1
+    filter: bool = False
 
 
 def more_route_plan(T, h, r, M, k, gate_mode=0, path=PATH_AUTO, msplit=0) -> RoutePlan:
@@ -96,6 +102,14 @@ def more_route_plan(T, h, r, M, k, gate_mode=0, path=PATH_AUTO, msplit=0) -> Rou
     if rc != 0:
         raise MoreRouteError(rc, "more_route_plan")
     return RoutePlan(a.value, b.value, c.value)
+
+
+def more_route_plan_ex(T, h, r, M, k, gate_mode=0, want_lse=False, path=PATH_AUTO, msplit=0) -> RoutePlan:
+    o = (ctypes.c_int * 7)()
+    rc = lib().more_route_plan_ex(T, h, r, M, k, gate_mode, int(want_lse), path, msplit, o)
+    if rc != 0:
+        raise MoreRouteError(rc, "more_route_plan_ex")
+    return RoutePlan(o[0], o[1], o[2], o[3], o[4], o[5], bool(o[6]))
 
 
 def _ptr(t):

@@ -7,7 +7,8 @@ import subprocess
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libmore_route.so")
-SOURCES = ["more_route_api.cu", "more_route_generic.cu", "more_route_sm100.cu", "more_route_noalloc.cu",
+SOURCES = ["more_route_api.cu", "more_route_generic.cu", "more_route_sm100.cu", "more_route_full_sm100.cu",
+           "more_route_noalloc.cu",
            "more_dispatch.cu", "more_psum_sm100.cu", "more_merge.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

@@ -34,6 +34,8 @@ struct DeviceCtx {
     unsigned long long* stats = nullptr;   // 16 diagnostic counters, next to the status word
     void* staging = nullptr;      // device staging of more_route_host
     size_t staging_bytes = 0;
+    float* colnorm_max = nullptr;       // device float: largest column norm of R2, written by the filter's preparation
+    unsigned* prep_arrivals = nullptr;  // device counter of that kernel (returns to zero after every launch)
 };
 
 // Largest number of tokens per CTA of the tensor-core path (rows of one X tile), and the expert-tile width.
@@ -46,19 +48,29 @@ struct Plan {
     int msplit;   // CTAs per token block
     int ctas;     // CTAs of the main kernel
     int rpad;     // r rounded up to a multiple of 16 (tensor-core path)
-    int block_tokens;   // tokens per CTA (tensor-core path): multiple of 32, <= kBlockTokens
+    int block_tokens;   // tokens per CTA (tensor-core path): a multiple of 32
+    int tg = 1;   // low-rank router: 128-token groups per CTA ...
+    int es = 1;   // ... and expert ranges swept side by side inside a CTA (tg * es <= 4)
+    bool filter = false;   // low-rank router: approximate sweep + exact rescoring of the survivors
 };
 
 bool tcgen05_shape_ok(int T, int h, int r, int M, int k);
-int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int sm_count, Plan* out);
+// want_lse: the caller asked for out_lse or the full-softmax gate; full: the standard (full-rank) router.
+int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, bool full, int path, int msplit,
+              int sm_count, Plan* out);
+bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st1_bytes, int* nst2, int* st2_bytes,
+                       int* r2_off);
 
 // Scratch bytes each path needs for a problem.
 size_t generic_scratch_bytes(const RouteArgs& a);
-size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p);
+size_t lowrank_scratch_bytes(const RouteArgs& a, const Plan& p);
+size_t full_scratch_bytes(const RouteArgs& a, const Plan& p);
 
 // Launchers: enqueue on a.stream, return MORE_OK / MORE_ERR_*.  `scratch` is at least *_scratch_bytes().
 int launch_generic(const RouteArgs& a, DeviceCtx& ctx, void* scratch);
-int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
+// Both tensor-core launchers clear out_counts on the stream themselves, after every host-side step that can fail.
+int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
+int launch_full(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
 
 int launch_generic_psum(const __nv_bfloat16* X, const __nv_bfloat16* R1, const __nv_bfloat16* R2, int T, int h, int r,
                         int M, const float* lse, float* psum, void* scratch, cudaStream_t stream);

@@ -4,6 +4,8 @@
 #include <atomic>
 #include <mutex>
 #include <new>
+#include <stdio.h>
+#include <stdlib.h>
 
 namespace more {
 
@@ -26,10 +28,12 @@ int get_ctx(DeviceCtx** out)
         c.cc_major = major;
         c.sm_count = sms;
         if (major != 10) return MORE_ERR_ARCH;
-        void* blk = nullptr;                   // status word + 16 diagnostic counters
+        void* blk = nullptr;                   // status word, the filter's two words, 16 diagnostic counters
         if (cudaMalloc(&blk, 256) != cudaSuccess) return MORE_ERR_CUDA;
         if (cudaMemset(blk, 0, 256) != cudaSuccess) return MORE_ERR_CUDA;
         c.status = static_cast<int*>(blk);
+        c.colnorm_max = reinterpret_cast<float*>(static_cast<char*>(blk) + 64);
+        c.prep_arrivals = reinterpret_cast<unsigned*>(static_cast<char*>(blk) + 68);
         c.stats = reinterpret_cast<unsigned long long*>(static_cast<char*>(blk) + 128);
         c.dev = dev;
     }
@@ -63,7 +67,8 @@ int check_shape(int T, int h, int r, int M, int k, int gate_mode, int path)
 
 bool aligned(const void* p, uintptr_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
 
-int route_device(const RouteArgs& a, int path, int msplit)
+// The body of every routing entry point.  The caller holds g_mutex.
+int route_device_locked(const RouteArgs& a, int path, int msplit)
 {
     int rc = check_shape(a.T, a.h, a.r, a.M, a.k, a.gate_mode, path);
     if (rc != MORE_OK) return rc;
@@ -74,59 +79,49 @@ int route_device(const RouteArgs& a, int path, int msplit)
         !aligned(a.out_lse, 4))
         return MORE_ERR_ALIGN;
 
-    std::lock_guard<std::mutex> lock(g_mutex);
     DeviceCtx* ctx = nullptr;
     rc = get_ctx(&ctx);
     if (rc != MORE_OK) return rc;
     Plan plan;
-    rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, path, msplit, ctx->sm_count, &plan);
+    const bool want_lse = a.gate_mode == MORE_GATE_FULL_SOFTMAX || a.out_lse != nullptr;
+    rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, want_lse, a.full, path, msplit, ctx->sm_count, &plan);
     if (rc != MORE_OK) return rc;
-    const size_t need = plan.path == MORE_PATH_TCGEN05 ? tcgen05_scratch_bytes(a, plan) : generic_scratch_bytes(a);
+    const size_t need = plan.path != MORE_PATH_TCGEN05 ? generic_scratch_bytes(a)
+                                                       : (a.full ? full_scratch_bytes(a, plan) : lowrank_scratch_bytes(a, plan));
     rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, need);
     if (rc != MORE_OK) return rc;
-    if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) return MORE_ERR_CUDA;
-    if (a.T == 0) return MORE_OK;
-    return plan.path == MORE_PATH_TCGEN05 ? launch_tcgen05(a, *ctx, plan, ctx->scratch)
-                                          : launch_generic(a, *ctx, ctx->scratch);
+    if (a.T == 0 || plan.path != MORE_PATH_TCGEN05) {
+        // (the tensor-core launchers clear out_counts themselves, after their last step that can fail)
+        if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) return MORE_ERR_CUDA;
+        if (a.T == 0) return MORE_OK;
+        return launch_generic(a, *ctx, ctx->scratch);
+    }
+    return a.full ? launch_full(a, *ctx, plan, ctx->scratch) : launch_lowrank(a, *ctx, plan, ctx->scratch);
+}
+
+int route_device(const RouteArgs& a, int path, int msplit)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    return route_device_locked(a, path, msplit);
 }
 
 }  // namespace
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
-int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int sm_count, Plan* out)
+namespace {
+
+// Launch plan of the fused standard router (256-token CTAs, two per SM).
+void plan_full(int T, int h, int M, int msplit, int sm_count, Plan* p)
 {
-    (void)gate_mode;
-    const bool fast_ok = tcgen05_shape_ok(T, h, r, M, k);
-    if (path == MORE_PATH_TCGEN05 && !fast_ok) return MORE_ERR_SHAPE;
-    if (msplit < 0) return MORE_ERR_SHAPE;
-    Plan p;
-    p.rpad = (r + 15) / 16 * 16;
-    if (path == MORE_PATH_GENERIC || !fast_ok) {
-        p.path = MORE_PATH_GENERIC;
-        p.block_tokens = 8;
-        p.msplit = 1;
-        p.ctas = (T + 7) / 8;
-        *out = p;
-        return MORE_OK;
-    }
-    p.path = MORE_PATH_TCGEN05;
-    if (sm_count <= 0) sm_count = 148;
     const int slots = 2 * sm_count;                       // two CTAs are resident per SM
     const int tiles = (M + kTileExperts - 1) / kTileExperts;
-    // Fill one wave of resident CTAs as evenly as possible.  Candidates: tokens per CTA (a multiple of 32 up to
-    // 256; smaller blocks waste rows of the second accumulator but even out the SMs) x CTAs per token block
-    // (each extra CTA repeats the block's z projection and starts its top-k from scratch, and a second, partial
-    // wave costs more than it gains; every CTA keeps at least eight expert tiles -- the first few hundred experts
-    // of a sweep cost far more than the rest, so short sweeps are not worth starting twice).
     double best = 1e300;
     int best_bt = kBlockTokens, best_s = 1;
     for (int bt = kBlockTokens; bt >= 128; bt -= 32) {
         const int blocks = (T + bt - 1) / bt;
         int s = msplit;
         if (s == 0) {
-            // while the CTAs have an SM each, splitting is cheap: keep eight tiles per CTA; once two CTAs share an
-            // SM the second one gains less than its repeated start costs: keep sixteen
             s = slots / blocks;
             if (s > tiles / 8) s = tiles / 8;
             if ((long long)blocks * s > sm_count) {
@@ -140,17 +135,107 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int ms
         }
         if (s > tiles) s = tiles;
         const long long ctas = (long long)blocks * s;
-        // makespan ~ (CTAs the busiest SM gets) x (time of one CTA); one CTA costs its projection (the X tile always
-        // has 256 rows), its share of the sweep (proportional to its live token rows) and a start-up term
         const double per_sm = (double)((ctas + sm_count - 1) / sm_count);
         const double per_cta = 256.0 * (h / 8.0) + (double)bt * ((double)tiles / s) * 16.0 + 256.0 * 256.0;
         const double cost = per_sm * per_cta;
         if (cost < best * 0.999) { best = cost; best_bt = bt; best_s = s; }
     }
-    if (best_s > 64) return MORE_ERR_SHAPE;
-    p.block_tokens = best_bt;
-    p.msplit = best_s;
-    p.ctas = ((T + best_bt - 1) / best_bt) * best_s;
+    p->block_tokens = best_bt;
+    p->msplit = best_s;
+    p->ctas = ((T + best_bt - 1) / best_bt) * best_s;
+}
+
+// Launch plan of the low-rank router: one CTA per SM with four 128-lane groups, laid out as tg token groups x es expert
+// ranges; msplit CTAs per token block.  A rough cycle model picks among the candidates: a sweep's time per 16-column
+// chunk is the larger of one warp's latency chain and the issue slots of the warps that share a scheduler (one per
+// group), every sweep pays a start-up worth ~160 chunks (nearly every early logit is a candidate), the projection is
+// bounded by the SM's share of HBM bandwidth, and a second wave of CTAs costs a whole CTA time.
+void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, int sm_count, Plan* p)
+{
+    const int blocks64 = (M + 63) / 64;
+    const int rpad = r <= 16 ? 16 : (r <= 32 ? 32 : 64);
+    const bool filter_ok = !want_lse && k <= 16 && M >= 4096;
+    const double c_lat = want_lse ? 260.0 : 190.0, c_iss = want_lse ? 120.0 : 62.0;
+    double best = 1e300;
+    Plan bp = *p;
+    for (int bt = 512; bt >= 32; bt -= 32) {
+        const int blocks = (T + bt - 1) / bt;
+        const int tg = (bt + 127) / 128;
+        for (int es = 1; es * tg <= 4; es *= 2) {
+            if (es > 1 && blocks64 < es * 4) continue;
+            int n1, b1, n2, b2, off;
+            if (!lowrank_smem_plan(rpad, tg, es, filter_ok, &n1, &b1, &n2, &b2, &off)) continue;
+            int s_lo = 1, s_hi = 1;
+            if (msplit > 0) {
+                s_lo = s_hi = msplit;
+            } else {
+                s_hi = sm_count / blocks;                      // never more CTAs than one wave
+                if (s_hi > blocks64 / (es * 8)) s_hi = blocks64 / (es * 8);    // a range keeps at least 512 experts
+                if (s_hi > 64) s_hi = 64;
+                if (s_hi < 1) s_hi = 1;
+            }
+            for (int s = s_lo; s <= s_hi; ++s) {
+                if ((long long)s * es > blocks64) continue;
+                const long long ctas = (long long)blocks * s;
+                const double waves = (double)((ctas + sm_count - 1) / sm_count);
+                const double chunks = 4.0 * blocks64 / (es * s) + 160.0;
+                const double groups = (double)tg * es;                      // warps per scheduler
+                const double per_chunk = c_lat > groups * c_iss ? c_lat : groups * c_iss;
+                const double ktile = bt * 128.0 / 23.0 > 300.0 ? bt * 128.0 / 23.0 : 300.0;
+                double t = 9000.0 + ((h + 63) / 64) * ktile + chunks * per_chunk;
+                if (es > 1) t += 1500.0;
+                if (s > 1) t += 7000.0 + 60.0 * s;
+                const double cost = waves * t;
+                if (cost < best * 0.999) {
+                    best = cost;
+                    bp.block_tokens = bt; bp.tg = tg; bp.es = es; bp.msplit = s; bp.ctas = (int)ctas;
+                }
+            }
+        }
+    }
+    *p = bp;
+    p->filter = filter_ok;
+}
+
+}  // namespace
+
+int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, bool full, int path, int msplit,
+              int sm_count, Plan* out)
+{
+    (void)gate_mode;
+    const bool fast_ok = tcgen05_shape_ok(T, h, r, M, k);
+    if (path == MORE_PATH_TCGEN05 && !fast_ok) return MORE_ERR_SHAPE;
+    if (msplit < 0 || msplit > 64) return MORE_ERR_SHAPE;
+    Plan p;
+    p.rpad = (r + 15) / 16 * 16;
+    if (path == MORE_PATH_GENERIC || !fast_ok) {
+        p.path = MORE_PATH_GENERIC;
+        p.block_tokens = 8;
+        p.msplit = 1;
+        p.ctas = (T + 7) / 8;
+        *out = p;
+        return MORE_OK;
+    }
+    p.path = MORE_PATH_TCGEN05;
+    if (sm_count <= 0) sm_count = 148;
+    if (full) {
+        plan_full(T, h, M, msplit, sm_count, &p);
+    } else {
+        p.block_tokens = 0;
+        plan_lowrank(T, h, r, M, k, want_lse, msplit, sm_count, &p);
+        if (p.block_tokens == 0) return MORE_ERR_SHAPE;
+#ifdef MORE_DEV
+        // development builds only: MORE_PLAN="block_tokens,es,msplit,filter" overrides the planner
+        if (const char* e = getenv("MORE_PLAN")) {
+            int bt = 0, es = 0, s = 0, f = 0;
+            if (sscanf(e, "%d,%d,%d,%d", &bt, &es, &s, &f) == 4) {
+                p.block_tokens = bt; p.tg = (bt + 127) / 128; p.es = es; p.msplit = s;
+                p.filter = f != 0 && !want_lse && k <= 16;
+                p.ctas = ((T + bt - 1) / bt) * s;
+            }
+        }
+#endif
+    }
     *out = p;
     return MORE_OK;
 }
@@ -211,16 +296,15 @@ int more_route_host(const void* Xh, const void* R1h, const void* R2h, int T, int
     auto up = [](size_t b) { return (b + 255) & ~(size_t)255; };
     const size_t bX = up((size_t)T * h * 2), bR1 = up((size_t)h * r * 2), bR2 = up((size_t)r * M * 2);
     const size_t bI = up((size_t)T * k * 4), bG = up((size_t)T * k * 4), bC = up((size_t)M * 4);
-    char* base = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(g_mutex);
-        DeviceCtx* ctx = nullptr;
-        rc = get_ctx(&ctx);
-        if (rc != MORE_OK) return rc;
-        rc = ensure_bytes(&ctx->staging, &ctx->staging_bytes, bX + bR1 + bR2 + bI + bG + bC);
-        if (rc != MORE_OK) return rc;
-        base = static_cast<char*>(ctx->staging);
-    }
+    // The staging buffer is shared by every call on the device and may be reallocated by a larger one, so the mutex
+    // is held until this call's copies and kernels have finished with it (the call synchronises the stream anyway).
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    rc = ensure_bytes(&ctx->staging, &ctx->staging_bytes, bX + bR1 + bR2 + bI + bG + bC);
+    if (rc != MORE_OK) return rc;
+    char* base = static_cast<char*>(ctx->staging);
     char* dX = base; char* dR1 = dX + bX; char* dR2 = dR1 + bR1;
     char* dI = dR2 + bR2; char* dG = dI + bI; char* dC = dG + bG;
     bool ok = true;
@@ -230,8 +314,16 @@ int more_route_host(const void* Xh, const void* R1h, const void* R2h, int T, int
         ok = ok && cudaMemcpyAsync(dR2, R2h, (size_t)r * M * 2, cudaMemcpyHostToDevice, st) == cudaSuccess;
     }
     if (!ok) return MORE_ERR_CUDA;
-    rc = more_route(dX, dR1, dR2, T, h, r, M, k, gate_mode, reinterpret_cast<int32_t*>(dI),
-                    reinterpret_cast<float*>(dG), reinterpret_cast<int32_t*>(dC), stream);
+    RouteArgs a;
+    a.X = reinterpret_cast<const __nv_bfloat16*>(dX);
+    a.R1 = reinterpret_cast<const __nv_bfloat16*>(dR1);
+    a.R2 = reinterpret_cast<const __nv_bfloat16*>(dR2);
+    a.T = T; a.h = h; a.r = r; a.M = M; a.k = k; a.gate_mode = gate_mode;
+    a.out_idx = reinterpret_cast<int32_t*>(dI); a.out_gate = reinterpret_cast<float*>(dG);
+    a.out_counts = reinterpret_cast<int32_t*>(dC);
+    a.out_topval = nullptr; a.out_lse = nullptr;
+    a.stream = st;
+    rc = route_device_locked(a, MORE_PATH_AUTO, 0);
     if (rc != MORE_OK) return rc;
     if (T > 0) {
         ok = ok && cudaMemcpyAsync(idx_h, dI, (size_t)T * k * 4, cudaMemcpyDeviceToHost, st) == cudaSuccess;
@@ -291,17 +383,30 @@ int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M
                            static_cast<cudaStream_t>(stream));
 }
 
-int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int* path_out,
-                    int* msplit_out, int* ctas_out)
+int more_route_plan_ex(int T, int h, int r, int M, int k, int gate_mode, int want_lse, int path, int msplit,
+                       int* out7)
 {
     int rc = check_shape(T, h, r, M, k, gate_mode, path);
     if (rc != MORE_OK) return rc;
+    if (!out7) return MORE_ERR_NULL;
     Plan p;
-    rc = make_plan(T, h, r, M, k, gate_mode, path, msplit, 148, &p);
+    rc = make_plan(T, h, r, M, k, gate_mode, want_lse != 0 || gate_mode == MORE_GATE_FULL_SOFTMAX, false, path, msplit,
+                   148, &p);
     if (rc != MORE_OK) return rc;
-    if (path_out) *path_out = p.path;
-    if (msplit_out) *msplit_out = p.msplit;
-    if (ctas_out) *ctas_out = p.ctas;
+    out7[0] = p.path; out7[1] = p.msplit; out7[2] = p.ctas; out7[3] = p.block_tokens;
+    out7[4] = p.tg; out7[5] = p.es; out7[6] = p.filter ? 1 : 0;
+    return MORE_OK;
+}
+
+int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int* path_out,
+                    int* msplit_out, int* ctas_out)
+{
+    int o[7];
+    const int rc = more_route_plan_ex(T, h, r, M, k, gate_mode, 0, path, msplit, o);
+    if (rc != MORE_OK) return rc;
+    if (path_out) *path_out = o[0];
+    if (msplit_out) *msplit_out = o[1];
+    if (ctas_out) *ctas_out = o[2];
     return MORE_OK;
 }
 

@@ -1,40 +1,42 @@
-// Tensor-core path of the fused low-rank router for sm_100a: TMA-staged operands, tcgen05.mma with TMEM
-// accumulators, a thread-per-token epilogue that keeps the running top-k (and, on request, the online
-// (max, sum-of-exponentials) pair of Eq. app_online) in registers.
+// Tensor-core path of the fused low-rank router for sm_100a (Algorithm 1 with the gates of Section 2 / Eq. app_softmax
+// and the per-expert counts fused in).  One CTA per SM, 18 warps:
 //
-// One CTA routes one block of 256 tokens (two 128-row accumulators) over one contiguous range of expert tiles
-// (Algorithm 1, with the token block additionally split over `msplit` CTAs along the expert dimension):
+//   warp 0       TMA producer: X and R1 k-tiles for phase 1, R2 blocks of 64 experts for phase 2.
+//   warp 1       tensor-memory allocation and tcgen05.mma issue (the warp stays converged, one elected lane issues).
+//   warps 2..17  epilogue: four groups of four warps.  A group owns 128 tensor-memory lanes = 128 tokens and one
+//                contiguous range of experts; a thread owns one token of its group.
 //
-//   phase 1  z = X_blk R1            TMA streams 256x64 X tiles (128x64 and twice the stages for blocks of at most 128
-//                                    tokens) and 64x64 R1 tiles (zero-filled beyond r), tcgen05.mma accumulates two
-//                                    128 x 64 fp32 blocks in TMEM.
-//   narrow   z -> bf16 hi + bf16 lo  written back to tensor memory (tcgen05.st) as the A operands [hi | lo] of phase 2:
-//                                    TMEM lane = token, two K-elements per 32-bit column.  Carrying both parts keeps
-//                                    the logits within ~3e-5 of exact arithmetic.
-//   phase 2  y = z R2[:, block]      64 experts at a time: TMA brings the r x 64 block of R2 once for both
-//                                    accumulators, tcgen05.mma with A from tensor memory (hi then lo into the same
-//                                    accumulator) fills 64 TMEM columns, the epilogue drains them: each epilogue
-//                                    thread owns one token and reads its logits 16 columns at a time.  The group hands
-//                                    the accumulator back as soon as the last 32 columns are in registers, so the next
-//                                    step's MMAs run while those are processed.
-//   merge    running top-k           sorted (value, id) list in registers, fed through a per-token candidate buffer
-//                                    in shared memory (see Selector).
-//   finish   gates, ids, counts      written by the CTA itself (msplit == 1) or, after the partial lists have been
-//                                    parked in scratch, by whichever CTA of the token block finishes last.
+// A CTA routes `block_tokens` (<= 512) tokens.  Its four groups are laid out as tg token groups x es expert ranges
+// (tg * es <= 4): with many tokens per SM every group takes different tokens and sweeps all of the CTA's experts; with
+// few tokens per SM several groups share the same 128 tokens and sweep different expert ranges, and their lists are
+// merged through shared memory at the end.  On top of that a token block can be split over `msplit` CTAs along the
+// expert axis (partial lists parked in global scratch, merged by the CTA that finishes last).
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM allocation + MMA issue (the whole warp stays converged and one
-// elected lane issues; see tc_mma_bf16_ts_elect), warps 2..9 = epilogue (warp w reads TMEM lanes 32*(w%4).. of
-// accumulator (w-2)/4).  Two CTAs are resident per SM (256 TMEM columns and ~112 KB of shared memory each): while one
-// group's epilogue drains its accumulator the MMAs of the other three groups of the SM run.  The same kernel with
-// FULL = true is the fused standard router (no z; every step contracts over all of h).
+//   phase 1  z = X_blk R1            128 x 64 X tiles and 64 x 64 R1 tiles by TMA, tcgen05.mma into fp32 accumulators.
+//   narrow   z -> bf16 operand       each group writes z into its own tensor-memory columns as the A operand of
+//                                    phase 2 (tcgen05.st): bf16 high part + bf16 low part in the exact modes, the high
+//                                    part alone in filter mode.
+//   phase 2  y = z R2[:, 32 experts] N = 32 MMAs with A from tensor memory fill a ring of 32-column accumulators per
+//                                    group (three, or two when the operand needs 64 columns); the epilogue warps drain
+//                                    them 16 columns at a time and hand each buffer back as soon as it is in registers,
+//                                    so the MMAs run up to a ring ahead of the slowest warp of a group.
+//   select   running top-k           sorted list in registers fed through a per-token candidate buffer in shared
+//                                    memory (Selector).
+//   finish   gates, ids, counts.
 //
-// Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
-// status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
+// Filter mode (top-k-softmax gate, no log-sum-exp wanted).  The second contraction runs on the high part of z only,
+// which halves its tensor work and frees tensor memory for the ring, but perturbs each logit by up to
+// E = |z - hi(z)|_2 * max_j |R2[:, j]|_2 (Cauchy-Schwarz; about 1e-2).  The sweep therefore keeps, besides the running
+// top-k of the approximate logits, every expert within W = 2E below the k-th of them (the "zone": any expert of the
+// true top-k lies there), and the survivors' logits are then recomputed in fp32 from the full z and the expert's
+// column (a row of the transposed copy of R2 the preparation kernel writes), which decides the final top-k, order
+// and gates.  A token whose zone overflows its few slots is routed again by a plain CUDA-core sweep at the end, so
+// the result is always the exact top-k of the fp32 logits.
+//
+// Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device status
+// word, raises the CTA's abort flag and all roles fall through to the common exit (tensor memory is freed there).
 #include "sm100_common.cuh"
 
-#include <limits.h>
-
-// -DMORE_STATS builds count epilogue events and clocks into KernelParams::stats (diagnostics only).
 #ifdef MORE_STATS
 #define STAT(...) __VA_ARGS__
 #else
@@ -45,107 +47,163 @@ namespace more {
 
 namespace {
 
-// -------------------------------------------------------------------------------------------- running top-k
-template <int KCAP>
-struct TopList {
-    float v[KCAP];
-    int id[KCAP];
-    __device__ __forceinline__ void init()
-    {
-#pragma unroll
-        for (int s = 0; s < KCAP; ++s) { v[s] = -INFINITY; id[s] = INT_MAX; }
-    }
-    __device__ __forceinline__ float tau() const { return v[KCAP - 1]; }
-    // Insert (x, j) with x > tau().  Equal values keep the earlier (smaller-id) entry ahead.
-    __device__ __forceinline__ void insert(float x, int j)
-    {
-#pragma unroll
-        for (int s = KCAP - 1; s > 0; --s) {
-            const bool above_prev = x > v[s - 1];
-            const bool above_this = x > v[s];
-            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
-            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
-        }
-        const bool top = x > v[0];
-        v[0] = top ? x : v[0];
-        id[0] = top ? j : id[0];
-    }
-    // Insert with the full order (value descending, id ascending): for merging lists whose ids interleave.
-    __device__ __forceinline__ void insert_ordered(float x, int j)
-    {
-        auto ahead = [&](int s) { return x > v[s] || (x == v[s] && j < id[s]); };
-#pragma unroll
-        for (int s = KCAP - 1; s > 0; --s) {
-            const bool above_prev = ahead(s - 1);
-            const bool above_this = ahead(s);
-            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
-            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
-        }
-        const bool top = ahead(0);
-        v[0] = top ? x : v[0];
-        id[0] = top ? j : id[0];
-    }
+constexpr int kGroups = 4;                         // 128-token groups per CTA
+constexpr int kEpiThreads = 128 * kGroups;
+constexpr int kRThreads = 64 + kEpiThreads;        // warps 0, 1 + 16 epilogue warps
+constexpr int kRRing = 208 * 1024;                 // shared-memory working area
+constexpr int kRSmem = kRRing + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
+constexpr int kGroupCols = 128;                    // tensor-memory columns per group
+constexpr int kBufCols = 32;                       // one accumulator buffer of the ring
+constexpr int kCandCap = 8;                        // candidate slots per token
+constexpr int kCandValStride = kEpiThreads * 16;   // bytes between successive value slots of one thread
+constexpr int kCandColStride = kEpiThreads * 4;    // ... and between its column slots
+constexpr int kCandValBytes = kCandCap * kCandValStride;
+constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);      // 80 KB
+constexpr int kZoneCap = 8;                        // zone slots per token (filter mode)
+constexpr int kZoneStride = kEpiThreads * 4;
+constexpr int kZoneIdOff = kZoneCap * kZoneStride;
+constexpr int kZoneBytes = 2 * kZoneIdOff;         // 32 KB
+constexpr int kXGroupBytes = 128 * 128;            // X tile of one token group: 128 tokens x 64 bf16
+constexpr int kR1Bytes = 64 * 128;
+constexpr int kFallbackSlots = 16;                 // tokens re-routed per round of the fallback (one per epilogue warp)
+constexpr unsigned kFullMask = 0xffffffffu;
+constexpr float kLog2e = 1.4426950408889634f;
+
+enum { kModeExact = 0, kModeExactLse = 1, kModeFilter = 2 };
+
+struct RouteParams {
+    int T, h, r, M, k, gate_mode;
+    int msplit, es, tg;          // CTAs per token block; expert ranges and token groups inside a CTA
+    int block_tokens;            // tokens per CTA: a multiple of 32, at most 128 * tg
+    int blocks64;                // ceil(M / 64)
+    int nst1, st1_bytes;         // phase-1 stages
+    int nst2, st2_bytes, r2_off; // phase-2 stages (es R2 blocks each) and where they start in the ring
+    int32_t* out_idx;
+    float* out_gate;
+    int32_t* out_counts;
+    float* out_topval;
+    float* out_lse;
+    int* status;
+    unsigned long long* stats;
+    // global scratch of an msplit > 1 launch: per token block an arrival counter, per (token, split) a partial list
+    unsigned* counters;
+    float* part_val;
+    int* part_id;
+    float2* part_mz;
+    // filter mode: transposed copy of R2 ([M][RPAD] bf16, columns >= r zero) and the largest column norm of R2
+    const __nv_bfloat16* r2t;
+    const float* colnorm_max;
+    const __nv_bfloat16* R2;     // for the fallback sweep
 };
 
-// Running top-k of one token.  Between refreshes the sorted list is left alone.  A chunk of 16 logits is looked at
-// as four groups of four; every group whose maximum beats the cached threshold `tau` (the list's last entry as of
-// the last refresh, hence never above the true threshold) is appended whole, in ascending column order, to this
-// thread's column of a shared-memory candidate buffer: one predicated 16-byte store of the four values (they sit in
-// four consecutive registers as loaded from tensor memory, so nothing is moved), one predicated 4-byte store of the
-// group's first column into a parallel array, and no branch.  refresh() then inserts the buffered elements that beat
-// the up-to-date threshold, so the inserts of several chunks of all 32 tokens of a warp are executed together.  A
-// chunk appends at most 4 entries and the warp refreshes as soon as some token has fewer than 4 free slots left, so
-// the buffer cannot overflow.
-constexpr int kCandValStride = kEpilogueThreads * 16;     // bytes between successive value slots of one thread
-constexpr int kCandColStride = kEpilogueThreads * 4;      // ... and between its column slots
-#ifndef MORE_CAND_CAP
-#define MORE_CAND_CAP 8
-#endif
-constexpr unsigned kFullMask = 0xffffffffu;
+// ---------------------------------------------------------------------------------------- shared-memory access
+__device__ __forceinline__ float lds_f32(uint32_t a)
+{
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ int lds_s32(uint32_t a)
+{
+    int v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
+    return v;
+}
+__device__ __forceinline__ void sts_f32(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
+__device__ __forceinline__ void sts_s32(uint32_t a, int v) { asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
+__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
 
-template <int KCAP, int CAP>
+// Running top-k of one token.  Between folds the sorted list is left alone.  A chunk of 16 logits is looked at as four
+// groups of four; every group whose maximum beats the cached threshold `thr` (never above the true one) is appended
+// whole, in ascending column order, to this thread's column of a shared-memory candidate buffer: one predicated
+// 16-byte store of the four values (they sit in four consecutive registers as loaded from tensor memory), one
+// predicated 4-byte store of the group's first column, no branch.  fold() then inserts the buffered elements that beat
+// the up-to-date threshold, so the inserts of several chunks of all 32 tokens of a warp are executed together.  A chunk
+// appends at most 4 entries and the warp folds as soon as some token has fewer than 4 free slots left, so the buffer
+// cannot overflow.
+//
+// FILTER: the logits are approximate to within E; thr sits W = 2E below the list's last value, elements that land in
+// that zone (directly, or pushed out of the list) are kept in a second small per-token store, pruned when it fills
+// up; a token whose zone still overflows is flagged for the fallback.
+template <int KCAP, bool FILTER>
 struct Selector {
-    static constexpr int kWarnSlots = CAP - 4;            // a chunk must always find 4 free slots
-    static_assert(kWarnSlots >= 1, "candidate buffer too small");
     TopList<KCAP> L;
-    float tau;
-    uint32_t ptr;     // shared-memory address of this thread's next free value slot
-    uint32_t cptr;    // ... and of the matching column slot
-    uint32_t base, cbase;
-    uint32_t warn;    // at or beyond this fill level the warp refreshes after the chunk
+    float thr;
+    float W;
+    uint32_t ptr, cptr, base, cbase, warn;
+    uint32_t zptr, zbase;
+    bool overflow;
 
-    __device__ __forceinline__ void init(uint32_t first_val_slot, uint32_t first_col_slot)
+    __device__ __forceinline__ void init(uint32_t first_val_slot, uint32_t first_col_slot, uint32_t first_zone_slot, float w)
     {
         L.init();
-        tau = -INFINITY;
+        thr = -INFINITY;
+        W = w;
         base = ptr = first_val_slot;
         cbase = cptr = first_col_slot;
-        warn = first_val_slot + kWarnSlots * kCandValStride;
+        warn = first_val_slot + (kCandCap - 4) * kCandValStride;
+        zbase = zptr = first_zone_slot;
+        overflow = false;
     }
-    // Called by all 32 lanes of a warp together.  Every round inserts at most one element per token: the maximum
-    // of the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
-    // (rising) threshold any more moves on to its next entries.  The rounds end when no token has anything left, so
-    // their number is the largest count of real insertions of any token of the warp, and the (select-only) insert
-    // code is executed once per round.
-    __device__ __forceinline__ void refresh()
+    __device__ __forceinline__ float limit() const { return FILTER ? L.tau() - W : L.tau(); }
+
+    // Drop the zone entries that have fallen more than W below the list; flag the token if the zone is still full.
+    __device__ __forceinline__ void prune()
+    {
+        const float lim = limit();
+        uint32_t rd = zbase, wr = zbase;
+        while (__any_sync(kFullMask, rd < zptr)) {
+            const bool act = rd < zptr;
+            float v = -INFINITY;
+            int id = 0;
+            if (act) { v = lds_f32(rd); id = lds_s32(rd + kZoneIdOff); }
+            if (act && v > lim) {
+                sts_f32(wr, v);
+                sts_s32(wr + kZoneIdOff, id);
+                wr += kZoneStride;
+            }
+            rd += kZoneStride;
+        }
+        zptr = wr;
+        if (zptr >= zbase + kZoneCap * kZoneStride) { overflow = true; zptr = zbase; }
+    }
+
+    // Called by all 32 lanes of a warp together.  Every round handles at most one element per token: the maximum of
+    // the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
+    // (rising) limit any more moves on to its next entries.  The rounds end when no token has anything left.
+    __device__ __forceinline__ void fold()
     {
         uint32_t a = base, c = cbase;
         float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
         int col = 0;
         for (;;) {
             float m = fmaxf(max3(x0, x1, x2), x3);
-            while (!(m > L.tau()) && a < ptr) {
+            while (!(m > limit()) && a < ptr) {
                 asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(a) : "memory");
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(col) : "r"(c) : "memory");
+                col = lds_s32(c);
                 a += kCandValStride;
                 c += kCandColStride;
                 m = fmaxf(max3(x0, x1, x2), x3);
             }
-            const bool pass = m > L.tau();
+            const bool pass = m > limit();
             if (!__any_sync(kFullMask, pass)) break;
             // the maximum's lowest column on a tie, so that equal logits enter the list in ascending column order
             const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : ((x2 == m) ? 2 : 3));
-            if (pass) L.insert(m, col + j);
+            if constexpr (FILTER) {
+                const bool ins = pass && (m > L.tau());
+                const float ev = ins ? L.v[KCAP - 1] : m;          // what may belong into the zone: the entry pushed
+                const int ei = ins ? L.id[KCAP - 1] : col + j;     // out of the list, or the element itself
+                if (ins) L.insert(m, col + j);
+                if (pass && ev > limit()) {
+                    sts_f32(zptr, ev);
+                    sts_s32(zptr + kZoneIdOff, ei);
+                    zptr += kZoneStride;
+                }
+                if (__any_sync(kFullMask, zptr >= zbase + kZoneCap * kZoneStride)) prune();
+            } else {
+                if (pass) L.insert(m, col + j);
+            }
             x0 = (j == 0) ? -INFINITY : x0;
             x1 = (j == 1) ? -INFINITY : x1;
             x2 = (j == 2) ? -INFINITY : x2;
@@ -153,9 +211,9 @@ struct Selector {
         }
         ptr = base;
         cptr = cbase;
-        tau = L.tau();
+        thr = limit();
     }
-    // if (t > tau) append {v0, v1, v2, v3} and col
+    // if (t > thr) append {v0, v1, v2, v3} and col
     __device__ __forceinline__ void append4(float t, float v0, float v1, float v2, float v3, int col)
     {
         asm volatile(
@@ -166,7 +224,7 @@ struct Selector {
             "@p add.u32 %0, %0, %9;\n\t"
             "@p add.u32 %1, %1, %10;\n\t}"
             : "+r"(ptr), "+r"(cptr)
-            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "f"(v3), "r"(col), "f"(tau), "n"(kCandValStride), "n"(kCandColStride)
+            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "f"(v3), "r"(col), "f"(thr), "n"(kCandValStride), "n"(kCandColStride)
             : "memory");
     }
     // v: 16 logits of columns col0.., t: maxima of the groups (v[4i] .. v[4i+3]).
@@ -177,31 +235,12 @@ struct Selector {
     }
 };
 
-struct KernelParams {
-    int T, h, r, M, k, gate_mode, msplit;
-    int block_tokens;            // tokens routed per CTA: a multiple of 32, at most 256
-    int x_rows;                  // rows of the X tile: 256, or 128 when block_tokens <= 128 (low-rank router only)
-    int tiles_total;             // ceil(M / 128)
-    int32_t* out_idx;
-    float* out_gate;
-    int32_t* out_counts;
-    float* out_topval;
-    float* out_lse;
-    int* status;
-    unsigned long long* stats;   // diagnostic event counters (only written by -DMORE_STATS builds)
-    // scratch (msplit > 1): per token block an arrival counter, per (token, split) a partial list and (m, Z)
-    unsigned* counters;
-    float* part_val;
-    int* part_id;
-    float2* part_mz;
-};
-
 // Final outputs of one token from its sorted list and (m2, z): m2 is the running max in log2 units.
 template <int KCAP>
-__device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, const TopList<KCAP>& L, float m2,
+__device__ __forceinline__ void write_token(const RouteParams& p, int64_t row, const TopList<KCAP>& L, float m2,
                                             float zsum, int* hist)
 {
-    constexpr float kLn2 = 0.6931471805599453f, kLog2e = 1.4426950408889634f;
+    constexpr float kLn2 = 0.6931471805599453f;
     const int k = p.k;
     float denom = 0.f;
     if (p.gate_mode == MORE_GATE_TOPK_SOFTMAX) {
@@ -226,79 +265,110 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
     if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
 }
 
-// ------------------------------------------------------------------------------------------------- the kernel
-// FULL = true is the fused STANDARD router (logits = X W with W [h][M], no low-rank bottleneck: Alg. 1 without z, the
-// contraction running over K = h): there is no phase 1, every 64-expert step instead accumulates over all h/64 k-tiles
-// of X (256 x 64, re-read per step) and W (64 x 64) with the phase-1 pipeline and stage layout, and the epilogue is
-// the same.  map_r2 is then W's map (64 x 64 boxes), map_r1 is unused, RPAD is 64.
-template <int RPAD, int KCAP, bool LSE, bool FULL = false>
-__global__ void __launch_bounds__(kThreads, 2)
-route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
-                     const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
+// Exact top-KCAP of one token over experts [e_lo, e_hi) by a plain CUDA-core sweep, run by one warp: lane j takes the
+// experts e_lo + j, e_lo + j + 32, ..., computes each logit as the fp32 chain l = fma(z[i], R2[i][e], l) over i
+// ascending (the same chain the rescoring of the filter uses), keeps a lane-local sorted list, and the 32 lists are
+// merged by KCAP rounds of a warp-wide argmax under the full order (value descending, id ascending).  zs: the token's
+// z in shared memory (r floats); the result goes to out_v / out_id (shared memory, KCAP entries).
+template <int KCAP>
+__device__ __noinline__ void exact_topk_warp(const float* zs, const __nv_bfloat16* __restrict__ R2, int r, int M,
+                                             int e_lo, int e_hi, float* out_v, int* out_id, int lane)
 {
-    constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
-    constexpr int kHalf = 64;                                   // experts per phase-2 step: one 128-byte-wide R2 block
-    constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
-    // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
-    constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
-    using Sel = Selector<KCAP, kCandCap>;
-    constexpr int kCandValBytes = kCandCap * kCandValStride;
-    constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);
-    // R2 blocks in flight: what the ring has room for next to the candidate buffers, at most 8 (unused by FULL)
-    constexpr int kStagesFit = (kRingBytes - kCandBytes) / kR2StageBytes;
-    constexpr int kStagesP2 = FULL ? 1 : (kStagesFit < 8 ? kStagesFit : 8);
-    static_assert(FULL || kStagesP2 >= 2, "no room for the R2 pipeline");
-    constexpr int kCandOffset = FULL ? kStagesP1 * kP1StageBytes : 0;
-    static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRingBytes, "phase-2 layout does not fit");
-    // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
-    // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.
-    constexpr uint32_t kAccCols = 64, kZopCol0 = 128;
-    constexpr float kLog2e = 1.4426950408889634f;
+    TopList<KCAP> L;
+    L.init();
+    for (int e = e_lo + lane; e < e_hi; e += 32) {
+        float l = 0.f;
+        for (int i = 0; i < r; ++i) l = fmaf(zs[i], __bfloat162float(R2[(int64_t)i * M + e]), l);
+        if (l > L.tau()) L.insert(l, e);
+    }
+    for (int q = 0; q < KCAP; ++q) {
+        float bv = L.v[0];
+        int bi = L.id[0];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float ov = __shfl_xor_sync(kFullMask, bv, o);
+            const int oi = __shfl_xor_sync(kFullMask, bi, o);
+            const bool take = ov > bv || (ov == bv && oi < bi);
+            bv = take ? ov : bv;
+            bi = take ? oi : bi;
+        }
+        if (lane == 0) { out_v[q] = bv; out_id[q] = bi; }
+        if (L.id[0] == bi && L.v[0] == bv && bi != INT_MAX) {      // the winning lane pops its head
+#pragma unroll
+            for (int s = 0; s + 1 < KCAP; ++s) { L.v[s] = L.v[s + 1]; L.id[s] = L.id[s + 1]; }
+            L.v[KCAP - 1] = -INFINITY;
+            L.id[KCAP - 1] = INT_MAX;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------- the kernel
+template <int RPAD, int KCAP, int MODE>
+__global__ void __launch_bounds__(kRThreads, 1)
+route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
+                     const __grid_constant__ CUtensorMap map_r2, const RouteParams p)
+{
+    constexpr bool FILTER = MODE == kModeFilter;
+    constexpr bool LSE = MODE == kModeExactLse;
+    constexpr int kKSteps = RPAD / 16;                               // UMMA K = 16
+    constexpr int kMmasPerBuf = FILTER ? kKSteps : 2 * kKSteps;      // exact modes: hi then lo into one accumulator
+    constexpr int kZopCols = FILTER ? RPAD / 2 : RPAD;               // A operand: two bf16 per 32-bit column
+    constexpr int kRingCol0 = (kZopCols <= 32) ? 32 : 64;            // first column of the accumulator ring
+    constexpr int NBUF = (kGroupCols - kRingCol0) / kBufCols;        // 3 or 2
+    constexpr int kR2BlockBytes = RPAD * 128;                        // RPAD rows x 64 experts
+    constexpr int kZloOff = kCandBytes + kZoneBytes;                 // filter: low part of z, 16 B per (8 ranks, thread)
+    using Sel = Selector<KCAP, FILTER>;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;            // 1024-aligned: the 128-B swizzle repeats every 1 KB
     uint8_t* ring_ptr = smem_raw + (ring - raw);
-    uint8_t* ctl = ring_ptr + kRingBytes;                    // control block
+    uint8_t* ctl = ring_ptr + kRRing;                        // control block
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
-    // barrier slots
-    constexpr int kMaxStagesP1 = 4;
-    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kMaxStagesP1, B_ZACC = B_EMPTY1 + kMaxStagesP1, B_ZOP = B_ZACC + 1,
-                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
-                  B_COUNT = B_ACCE + 2;
+    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + 4, B_ZACC = B_EMPTY1 + 4, B_ZOP = B_ZACC + 1,
+                  B_FULL2 = B_ZOP + kGroups, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8,
+                  B_ACCE = B_ACCF + kGroups * 3, B_COUNT = B_ACCE + kGroups * 3;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
+    int* flagged = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 12);      // tokens that need the fallback sweep
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
-    STAT(const long long st_top = clock64();)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int blk = blockIdx.x / p.msplit, split = blockIdx.x % p.msplit;
     const int tok0 = blk * p.block_tokens;
-    // expert tiles of this CTA: an even share of ceil(M/128) tiles
-    const int tile_lo = (int)(((long long)p.tiles_total * split) / p.msplit);
-    const int tile_hi = (int)(((long long)p.tiles_total * (split + 1)) / p.msplit);
+    const int live_tokens = min(p.block_tokens, p.T - tok0);
+    const int tg_live = (live_tokens + 127) >> 7;            // token groups with at least one token
+    const int es = p.es;
+    const int ngroups = tg_live * es;
+    const int nparts = p.msplit * es;
+    // 64-expert blocks of expert range `esi` of this CTA: an even share of ceil(M / 64) blocks
+    auto part_lo = [&](int esi) { return (int)(((long long)p.blocks64 * (split * es + esi)) / nparts); };
+    auto part_hi = [&](int esi) { return (int)(((long long)p.blocks64 * (split * es + esi + 1)) / nparts); };
+    auto live_warps = [&](int tgi) { return min(4, (live_tokens - tgi * 128 + 31) >> 5); };
     const int ktiles1 = (p.h + 63) / 64;
-    // phase-1 stages: a 128-row X tile (small token blocks) leaves room for four k-tiles in flight instead of two,
-    // which matters when a CTA's projection is a chain of L2 round trips rather than a stream
-    const int x_tile_bytes = p.x_rows * 128;
-    const int st1_bytes = x_tile_bytes + kR1TileBytes;
-    const int nst1 = (p.x_rows == 128) ? 4 : kStagesP1;
+    int nsteps_max = 0;
+    for (int e = 0; e < es; ++e) nsteps_max = max(nsteps_max, part_hi(e) - part_lo(e));
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < kMaxStagesP1; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
         mbar_init(bar(B_ZACC), 1);
-        mbar_init(bar(B_ZOP), kEpilogueThreads);
+        for (int t = 0; t < kGroups; ++t) mbar_init(bar(B_ZOP + t), t < tg_live ? es * live_warps(t) : 1);
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads / 2); }
+        for (int g = 0; g < kGroups; ++g)
+            for (int s = 0; s < 3; ++s) {
+                mbar_init(bar(B_ACCF + g * 3 + s), 1);
+                mbar_init(bar(B_ACCE + g * 3 + s), g < ngroups ? live_warps(g / es) : 1);
+            }
         *abort_flag = 0;
         *last_flag = 0;
+        *flagged = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(kTmemCols)
+                     "r"(512)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -306,375 +376,516 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t cand = ring + kCandOffset;                   // phase 2: candidate buffers
-    const uint32_t r2ring = ring + kCandBytes;                  // phase 2: R2 stages
-    // 64-expert steps of this CTA (the last one of the last tile is skipped when it lies wholly beyond M)
-    const int e_lo = tile_lo * kTileExperts;
-    const int e_hi = min(tile_hi * kTileExperts, p.M);
-    const int nsteps = (e_hi - e_lo + kHalf - 1) / kHalf;
+    const uint32_t r2ring = ring + p.r2_off;
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
-        if (lane == 0 && FULL) {
-            // standard router: for every 64-expert step, all k-tiles of X and of W[:, step]
+        if (lane == 0) {
             bool ok = true;
-            const int total = nsteps * ktiles1;
-            for (int g = 0; g < total && ok; ++g) {
-                const int s = g % kStagesP1, it = g / ktiles1, kt = g % ktiles1;
-                if (g >= kStagesP1) ok = mbar_wait(bar(B_EMPTY1 + s), ((g / kStagesP1) - 1) & 1, abort_flag, p.status);
-                if (!ok) break;
-                const uint32_t dst = ring + s * kP1StageBytes;
-                mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
-                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // 256 token rows x 64 columns
-                tma_load_2d(dst + kXTileBytes, &map_r2, bar(B_FULL1 + s), e_lo + it * kHalf, kt * 64);
-            }
-        } else if (lane == 0) {
-            bool ok = true;
+            const uint32_t st1_tx = tg_live * kXGroupBytes + kR1Bytes;
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
-                const int s = kt % nst1;
-                if (kt >= nst1) ok = mbar_wait(bar(B_EMPTY1 + s), ((kt / nst1) - 1) & 1, abort_flag, p.status);
+                const int s = kt % p.nst1;
+                if (kt >= p.nst1) ok = mbar_wait(bar(B_EMPTY1 + s), ((kt / p.nst1) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t dst = ring + s * st1_bytes;
-                mbar_expect_tx(bar(B_FULL1 + s), st1_bytes);
-                tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // x_rows token rows x 64 columns
-                tma_load_2d(dst + x_tile_bytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
+                const uint32_t dst = ring + s * p.st1_bytes;
+                mbar_expect_tx(bar(B_FULL1 + s), st1_tx);
+                for (int t = 0; t < tg_live; ++t)                   // 128 token rows x 64 columns per token group
+                    tma_load_2d(dst + t * kXGroupBytes, &map_x, bar(B_FULL1 + s), kt * 64, tok0 + t * 128);
+                tma_load_2d(dst + p.tg * kXGroupBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
             }
-            // the ring is reused by phase 2: wait until every phase-1 MMA has finished reading it
-            ok = ok && mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
-            for (int it = 0; it < nsteps && ok; ++it) {
-                const int s = it % kStagesP2;
-                if (it >= kStagesP2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it / kStagesP2) - 1) & 1, abort_flag, p.status);
+            // the R2 stages lie beyond the phase-1 stages, so the first blocks of R2 arrive while phase 1 still runs
+            for (int it = 0; it < nsteps_max && ok; ++it) {
+                const int s = it % p.nst2;
+                if (it >= p.nst2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it / p.nst2) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                mbar_expect_tx(bar(B_FULL2 + s), kR2StageBytes);
-                tma_load_2d(r2ring + s * kR2StageBytes, &map_r2, bar(B_FULL2 + s), e_lo + it * kHalf, 0);
+                int nb = 0;
+                for (int e = 0; e < es; ++e) nb += (it < part_hi(e) - part_lo(e));
+                mbar_expect_tx(bar(B_FULL2 + s), nb * kR2BlockBytes);
+                for (int e = 0; e < es; ++e)
+                    if (it < part_hi(e) - part_lo(e))
+                        tma_load_2d(r2ring + s * p.st2_bytes + e * kR2BlockBytes, &map_r2, bar(B_FULL2 + s),
+                                    (part_lo(e) + it) * 64, 0);
             }
         }
     } else if (warp == 1) {
         // ======================================================================================= MMA issuer
         // The whole warp runs this code converged; one elected lane issues each tcgen05 instruction.
         bool ok = true;
-        constexpr uint32_t idesc1 = umma_idesc(64);
-        constexpr uint32_t idesc2 = umma_idesc(kHalf);
-        if constexpr (FULL) {
-            // standard router: per 64-expert step, K runs over all of h through the two k-tile stages
-            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), wd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
-            const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), w_lo0 = (uint32_t)wd, w_hi = (uint32_t)(wd >> 32);
-            int g = 0;
-            for (int it = 0; it < nsteps && ok; ++it) {
-                // both accumulators must have been read out (the k-tiles serve both token groups)
-#pragma unroll
-                for (int a = 0; a < 2; ++a)
-                    if (a * 128 < p.block_tokens)
-                        ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
-                if (!ok) break;
-                for (int kt = 0; kt < ktiles1 && ok; ++kt, ++g) {
-                    const int s = g % kStagesP1;
-                    ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (g / kStagesP1) & 1, abort_flag, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), w_lo = w_lo0 + s * (kP1StageBytes >> 4);
-#pragma unroll
-                    for (int a = 0; a < 2; ++a) {
-                        if (a * 128 >= p.block_tokens) continue;
-#pragma unroll
-                        for (int kk = 0; kk < 4; ++kk)
-                            tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
-                                                 w_lo + kk * (2048 >> 4), w_hi, idesc1, (kt | kk) != 0);
-                    }
-                    tc_commit_elect(bar(B_EMPTY1 + s));
-                }
-                if (!ok) break;
-#pragma unroll
-                for (int a = 0; a < 2; ++a)
-                    if (a * 128 < p.block_tokens) tc_commit_elect(bar(B_ACCF + a));
-            }
-        } else {
+        constexpr uint32_t idesc1 = umma_idesc(RPAD);
+        constexpr uint32_t idesc2 = umma_idesc(kBufCols);
         {
             // descriptor words of stage 0: K-major X tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address
-            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + x_tile_bytes, 8192, 1024);
+            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + p.tg * kXGroupBytes, 8192, 1024);
             const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
             for (int kt = 0; kt < ktiles1 && ok; ++kt) {
-                const int s = kt % nst1;
-                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / nst1) & 1, abort_flag, p.status));
+                const int s = kt % p.nst1;
+                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / p.nst1) & 1, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t x_lo = x_lo0 + s * (st1_bytes >> 4), r_lo = r_lo0 + s * (st1_bytes >> 4);
-#pragma unroll
-                for (int a = 0; a < 2; ++a) {
-                    if (a * 128 >= p.x_rows) continue;      // a 128-row X tile has no second token group
+                const uint32_t x_lo = x_lo0 + s * (p.st1_bytes >> 4), r_lo = r_lo0 + s * (p.st1_bytes >> 4);
+                for (int t = 0; t < tg_live; ++t) {
+                    // z of token group t accumulates in the ring columns of its first group
+                    const uint32_t d = tmem_base + (t * es) * kGroupCols + kRingCol0;
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
-                        tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
-                                             r_lo + kk * (2048 >> 4), r_hi, idesc1, (kt | kk) != 0);
+                        tc_mma_bf16_ss_elect(d, x_lo + t * (kXGroupBytes >> 4) + kk * 2, x_hi, r_lo + kk * (2048 >> 4),
+                                             r_hi, idesc1, (kt | kk) != 0);
                 }
                 tc_commit_elect(bar(B_EMPTY1 + s));
             }
         }
         if (ok) tc_commit_elect(bar(B_ZACC));
-        ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ZOP), 0, abort_flag, p.status));
+        // every group has written its operand (and, where groups share tokens, read the shared z) before phase 2
+        for (int t = 0; t < tg_live; ++t) ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ZOP + t), 0, abort_flag, p.status));
         tc_fence_after();
         const uint64_t bd0 = umma_desc_sw128(r2ring, 8192, 1024);
         const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
-        for (int it = 0; it < nsteps && ok; ++it) {
-            const int s = it % kStagesP2;
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status));
+        for (int it = 0; it < nsteps_max && ok; ++it) {
+            const int s = it % p.nst2;
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL2 + s), (it / p.nst2) & 1, abort_flag, p.status));
             if (!ok) break;
-            const uint32_t b_lo = b_lo0 + s * (kR2StageBytes >> 4);
 #pragma unroll
-            for (int a = 0; a < 2; ++a) {
-                if (a * 128 >= p.block_tokens) continue;     // a group without tokens takes no part in phase 2
-                // accumulator a is free once its 128 epilogue threads have read the previous step out of it
-                ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
+            for (int half = 0; half < 2; ++half) {
+                const int n = it * 2 + half;                         // the groups' n-th 32-expert buffer
+                const int slot = n % NBUF;
+                const uint32_t use = (uint32_t)(n / NBUF);
+                for (int g = 0; g < ngroups && ok; ++g) {
+                    const int esi = g % es;
+                    if (it >= part_hi(esi) - part_lo(esi)) continue;
+                    // the slot is free once the group's warps have read its previous contents out
+                    if (use > 0) ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCE + g * 3 + slot), (use - 1) & 1, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t d = tmem_base + g * kGroupCols + kRingCol0 + slot * kBufCols;
+                    const uint32_t a0 = tmem_base + g * kGroupCols;
+                    const uint32_t b_lo = b_lo0 + ((s * p.st2_bytes + esi * kR2BlockBytes) >> 4) + half * (64 >> 4);
 #pragma unroll
-                for (int j = 0; j < 2 * kKSteps; ++j)       // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
-                    tc_mma_bf16_ts_elect(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64 + j * 8,
-                                         b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
-                tc_commit_elect(bar(B_ACCF + a));
+                    for (int j = 0; j < kMmasPerBuf; ++j)       // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
+                        tc_mma_bf16_ts_elect(d, a0 + j * 8, b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
+                    tc_commit_elect(bar(B_ACCF + g * 3 + slot));
+                }
             }
             if (!ok) break;
             tc_commit_elect(bar(B_EMPTY2 + s));
         }
-        }   // !FULL
     } else {
         // ========================================================================================= epilogue
-        const int q = warp & 3;                              // TMEM lane group this warp may read
-        const int acc = (warp - 2) >> 2;                     // which 128-token accumulator
-        const int row_in_acc = q * 32 + lane;
-        const int row_in_blk = acc * 128 + row_in_acc;
+        const int ew = warp - 2;
+        const int g = ew >> 2;                               // group
+        const int q = warp & 3;                              // TMEM lane quarter this warp may access
+        const int etid = threadIdx.x - 64;                   // 0..511 among the epilogue threads
+        const int tgi = g / es, esi = g % es;
+        const int row_in_tg = q * 32 + lane;
+        const int row_in_blk = tgi * 128 + row_in_tg;
         const int64_t row = (int64_t)tok0 + row_in_blk;
-        const bool row_live = row_in_blk < p.block_tokens && row < p.T;     // rows past the block belong to the next CTA
-        const bool warp_live = acc * 128 + q * 32 < p.block_tokens;         // warp-uniform: block_tokens is a multiple of 32
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
-        const uint32_t t_zop = tmem_base + ((uint32_t)(q * 32) << 16) + kZopCol0 + acc * 64;
-        STAT(const long long st_k0 = clock64();)
-        bool ok = FULL ? true : mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
-        STAT(const long long st_k1 = clock64();)
-        if (ok && !FULL) {
-            // ---- narrow z to bf16 [hi | lo] and store it to tensor memory as the A operand of phase 2
+        const bool warp_live = g < ngroups && (tgi * 128 + q * 32) < live_tokens;     // warp-uniform
+        const bool row_live = warp_live && row_in_blk < live_tokens;
+        const uint32_t t_lanes = tmem_base + ((uint32_t)(q * 32) << 16);
+        const uint32_t t_zacc = t_lanes + (tgi * es) * kGroupCols + kRingCol0;       // the token group's z (fp32)
+        const uint32_t t_zop = t_lanes + g * kGroupCols;                              // this group's A operand
+        const uint32_t t_ring = t_zop + kRingCol0;
+        const uint32_t zlo_addr = ring + kZloOff + etid * 16;
+        const int e_lo = part_lo(esi) * 64;
+        const int e_hi = min(part_hi(esi) * 64, p.M);
+        const int nb = warp_live ? 2 * (part_hi(esi) - part_lo(esi)) : 0;             // 32-expert buffers to drain
+
+        float zone_w = 0.f;
+        bool ok = true;
+        if (warp_live) {
+            ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
+            ok = __all_sync(kFullMask, ok);
+        }
+        if (warp_live && ok) {
+            // ---- narrow z to bf16 and store it to tensor memory as the A operand of phase 2
             tc_fence_after();
+            float lo2 = 0.f, z2 = 0.f;
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
-                tmem_ld16(t_lane + c * 16, z);
+                tmem_ld16(t_zacc + c * 16, z);
                 tmem_ld_wait16(z);
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
                     const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
-                    const __nv_bfloat16 l0 = __float2bfloat16_rn(z[2 * e] - __bfloat162float(h0));
-                    const __nv_bfloat16 l1 = __float2bfloat16_rn(z[2 * e + 1] - __bfloat162float(h1));
+                    const float d0 = z[2 * e] - __bfloat162float(h0), d1 = z[2 * e + 1] - __bfloat162float(h1);
+                    const __nv_bfloat16 l0 = __float2bfloat16_rn(d0), l1 = __float2bfloat16_rn(d1);
                     hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
                     lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                    if (FILTER) {
+                        // the part of z the approximate logits do not see, and z itself (hi + lo, as it is rescored)
+                        lo2 = fmaf(d0, d0, lo2);
+                        lo2 = fmaf(d1, d1, lo2);
+                        z2 = fmaf(z[2 * e], z[2 * e], z2);
+                        z2 = fmaf(z[2 * e + 1], z[2 * e + 1], z2);
+                    }
                 }
                 tmem_st8(t_zop + c * 8, hi);
-                tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                if (FILTER) {
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zlo_addr + (2 * c) * (kEpiThreads * 16)),
+                                 "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zlo_addr + (2 * c + 1) * (kEpiThreads * 16)),
+                                 "r"(lo[4]), "r"(lo[5]), "r"(lo[6]), "r"(lo[7]) : "memory");
+                } else {
+                    tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                }
             }
             tmem_st_wait();
             tc_fence_before();
-            mbar_arrive(bar(B_ZOP));
+            warp_arrive(bar(B_ZOP + tgi), lane);
+            if (FILTER) {
+                // |approximate - fp32 logit| <= |z - hi|_2 |R2_j|_2 (the missing low part) + accumulation rounding of
+                // the two evaluations (bounded by 2^-18 |z|_2 |R2_j|_2, a generous multiple of fp32 epsilon).
+                const float cn = __ldg(p.colnorm_max);
+                const float e_bound = sqrtf(lo2) * cn * 1.001f + sqrtf(z2) * cn * 3.8147e-6f;
+                zone_w = 2.f * e_bound * 1.001f + 1e-30f;
+            }
         }
 
         Sel S;
-        S.init(cand + row_in_blk * 16, cand + kCandValBytes + row_in_blk * 4);
-        STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_rcall = 0, st_riter = 0; long long st_twait = 0, st_tproc = 0, st_tref = 0;
+        S.init(ring + etid * 16, ring + kCandValBytes + etid * 4, ring + kCandBytes + etid * 4, zone_w);
+        STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_fold = 0; long long st_twait = 0, st_tfold = 0;
              const long long st_t0 = clock64();)
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
 
-        // `ok` is kept warp-uniform from here on (tcgen05.ld, elect and the votes below need all 32 lanes).
-        ok = __all_sync(kFullMask, ok);
+        // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate scan
+        auto process = [&](float (&v)[16], int col0) {
+            if (col0 + 16 > p.M) {                           // ragged end of the expert axis (warp-uniform)
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (col0 + i >= p.M) v[i] = -INFINITY;
+            }
+            float t[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) t[i] = fmaxf(max3(v[4 * i], v[4 * i + 1], v[4 * i + 2]), v[4 * i + 3]);
+            const float cmax = fmaxf(max3(t[0], t[1], t[2]), t[3]);
+            if (LSE) {
+                const float c2 = cmax * kLog2e;
+                if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
+                float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 16; i += 4) {
+                    a0 += ex2f(fmaf(v[i], kLog2e, -m2));
+                    a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
+                    a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
+                    a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+                }
+                zsum += (a0 + a1) + (a2 + a3);
+            }
+            STAT(st_chunks++;)
+            if (__any_sync(kFullMask, cmax > S.thr)) {
+                STAT(st_hit++; const uint32_t mark = S.ptr;)
+                S.scan(v, t, col0);
+                STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
+                if (__any_sync(kFullMask, S.ptr >= S.warn)) {      // some token is about to run out of slots
+                    STAT(st_fold++; const long long tr0 = clock64();)
+                    S.fold();
+                    STAT(st_tfold += clock64() - tr0;)
+                }
+            }
+        };
 
-        const bool group_live = acc * 128 < p.block_tokens;
-        for (int it = 0; it < nsteps && ok && group_live; ++it) {
-            const int e0 = e_lo + it * kHalf;
-            const bool ragged = e0 + kHalf > p.M;
+        // ---- the sweep: buffer n of the group lives in ring slot n % NBUF
+        if (nb > 0 && ok) {
             float va[16], vb[16];
-            // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate scan
-            auto process = [&](float (&v)[16], int col0) {
-#ifdef MORE_EXP_NOPROC
-                return;
-#endif
-                if (ragged) {
+            STAT(const long long tw0 = clock64();)
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + g * 3), 0, abort_flag, p.status));
+            STAT(st_twait += clock64() - tw0;)
+            if (ok) {
+                tc_fence_after();
+                tmem_ld16(t_ring, va);
+            }
+            uint32_t ph = 0;
+            for (int n0 = 0; n0 < nb && ok; n0 += NBUF, ph ^= 1) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (col0 + i >= p.M) v[i] = -INFINITY;
-                }
-                float t[4];
-#pragma unroll
-                for (int i = 0; i < 4; ++i) t[i] = fmaxf(max3(v[4 * i], v[4 * i + 1], v[4 * i + 2]), v[4 * i + 3]);
-                const float cmax = fmaxf(max3(t[0], t[1], t[2]), t[3]);
-                if (LSE) {
-                    const float c2 = cmax * kLog2e;
-                    if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
-                    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-#pragma unroll
-                    for (int i = 0; i < 16; i += 4) {
-                        a0 += ex2f(fmaf(v[i], kLog2e, -m2));
-                        a1 += ex2f(fmaf(v[i + 1], kLog2e, -m2));
-                        a2 += ex2f(fmaf(v[i + 2], kLog2e, -m2));
-                        a3 += ex2f(fmaf(v[i + 3], kLog2e, -m2));
+                for (int s = 0; s < NBUF; ++s) {
+                    const int n = n0 + s;
+                    if (n < nb && ok) {
+                        const int col0 = e_lo + n * kBufCols;
+                        tmem_ld_wait16(va);
+                        tmem_ld16(t_ring + s * kBufCols + 16, vb);
+                        process(va, col0);
+                        tmem_ld_wait16(vb);
+                        tc_fence_before();
+                        warp_arrive(bar(B_ACCE + g * 3 + s), lane);          // the buffer is in registers: hand it back
+                        if (n + 1 < nb) {
+                            const int s1 = (s + 1) % NBUF;
+                            const uint32_t ph1 = (s + 1 == NBUF) ? (ph ^ 1) : ph;
+                            STAT(const long long tw1 = clock64();)
+                            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + g * 3 + s1), ph1, abort_flag, p.status));
+                            STAT(st_twait += clock64() - tw1;)
+                            if (ok) {
+                                tc_fence_after();
+                                tmem_ld16(t_ring + s1 * kBufCols, va);
+                            }
+                        }
+                        process(vb, col0 + 16);
                     }
-                    zsum += (a0 + a1) + (a2 + a3);
                 }
-                // Append this chunk's candidate groups (a warp-uniform branch around predicated stores), then fold
-                // the buffers into the lists if some token of the warp is running out of slots.
-                STAT(st_chunks++;)
-#ifdef MORE_EXP_NOSCAN
-                m2 = fmaxf(m2, cmax);
-                return;
-#endif
-                if (__any_sync(kFullMask, cmax > S.tau)) {
-                    STAT(st_hit++; const uint32_t mark = S.ptr;)
-                    S.scan(v, t, col0);
-                    STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
-                    if (__any_sync(kFullMask, S.ptr >= S.warn)) {
-                        // some token is about to run out of slots: fold now
-                        STAT(st_rcall++; const long long tr0 = clock64();)
-                        S.refresh();
-                        STAT(st_tref += clock64() - tr0;)
-                    }
+            }
+        }
+        if (warp_live) S.fold();
+        TopList<KCAP>& L = S.L;
+
+        if (FILTER && warp_live && ok) {
+            // ---- rescoring: fp32 logits of the list and of the zone from the full z = hi + lo and the experts'
+            // columns (rows of the transposed copy); the exact values decide the final order
+            S.prune();
+            const int zcount = (int)((S.zptr - S.zbase) / kZoneStride);
+            int zmax = zcount;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) zmax = max(zmax, __shfl_xor_sync(kFullMask, zmax, o));
+            float acc[KCAP];
+#pragma unroll
+            for (int e = 0; e < KCAP; ++e) acc[e] = 0.f;
+            auto z_chunk = [&](int c, float (&z8)[8]) {             // ranks 8c .. 8c+7 of this token's z
+                uint32_t h4[4], l4[4];
+                tmem_ld4(t_zop + c * 4, h4);
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(l4[0]), "=r"(l4[1]), "=r"(l4[2]), "=r"(l4[3])
+                             : "r"(zlo_addr + c * (kEpiThreads * 16)) : "memory");
+                tmem_ld_wait4(h4);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    z8[2 * e] = bf_lo(h4[e]) + bf_lo(l4[e]);
+                    z8[2 * e + 1] = bf_hi(h4[e]) + bf_hi(l4[e]);
                 }
             };
-            STAT(const long long tw0 = clock64();)
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
-            STAT(const long long tw1 = clock64(); st_twait += tw1 - tw0;)
-            if (!ok) break;
-            if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
-                mbar_arrive(bar(B_ACCE + acc));
-                continue;
+            auto dot8 = [&](float a, const float (&z8)[8], const uint4& w) {
+                a = fmaf(z8[0], bf_lo(w.x), a); a = fmaf(z8[1], bf_hi(w.x), a);
+                a = fmaf(z8[2], bf_lo(w.y), a); a = fmaf(z8[3], bf_hi(w.y), a);
+                a = fmaf(z8[4], bf_lo(w.z), a); a = fmaf(z8[5], bf_hi(w.z), a);
+                a = fmaf(z8[6], bf_lo(w.w), a); a = fmaf(z8[7], bf_hi(w.w), a);
+                return a;
+            };
+            const uint4* r2t = reinterpret_cast<const uint4*>(p.r2t);
+            for (int c = 0; c < RPAD / 8; ++c) {
+                float z8[8];
+                z_chunk(c, z8);
+#pragma unroll
+                for (int e = 0; e < KCAP; ++e) {
+                    if ((unsigned)L.id[e] < (unsigned)p.M) {
+                        const uint4 w = __ldg(r2t + (size_t)L.id[e] * (RPAD / 8) + c);
+                        acc[e] = dot8(acc[e], z8, w);
+                    }
+                }
             }
-            tc_fence_after();
-            // columns 0-31: the load of the next 16 columns is in flight while the current 16 are processed
-            tmem_ld16(t_lane, va);
-            tmem_ld_wait16(va);
-            tmem_ld16(t_lane + 16, vb);
-            process(va, e0);
-            tmem_ld_wait16(vb);
-            tmem_ld16(t_lane + 32, va);
-            process(vb, e0 + 16);
-            // columns 32-63: both halves are brought into registers first; the accumulator can then be handed back,
-            // and the next step's MMAs run while these 32 columns are processed
-            tmem_ld_wait16(va);
-            tmem_ld16(t_lane + 48, vb);
-            tmem_ld_wait16(vb);
-            tc_fence_before();
-            mbar_arrive(bar(B_ACCE + acc));
-            process(va, e0 + 32);
-            process(vb, e0 + 48);
-            STAT(st_tproc += clock64() - tw1;)
+            TopList<KCAP> F;
+            F.init();
+#pragma unroll
+            for (int e = 0; e < KCAP; ++e)
+                if ((unsigned)L.id[e] < (unsigned)p.M) F.insert_ordered(acc[e], L.id[e]);
+            for (int zi = 0; zi < zmax; ++zi) {
+                const bool have = zi < zcount;
+                const int id = have ? lds_s32(S.zbase + kZoneIdOff + zi * kZoneStride) : -1;
+                float a = 0.f;
+                for (int c = 0; c < RPAD / 8; ++c) {
+                    float z8[8];
+                    z_chunk(c, z8);
+                    if ((unsigned)id < (unsigned)p.M) a = dot8(a, z8, __ldg(r2t + (size_t)id * (RPAD / 8) + c));
+                }
+                if ((unsigned)id < (unsigned)p.M) F.insert_ordered(a, id);
+            }
+            L = F;
         }
-        S.refresh();
-        TopList<KCAP>& L = S.L;
 #ifdef MORE_STATS
-        if (lane == 0 && p.stats) {
+        if (lane == 0 && p.stats && warp_live) {
             atomicAdd(p.stats + 0, (unsigned long long)st_chunks);
             atomicAdd(p.stats + 1, (unsigned long long)st_hit);
             atomicAdd(p.stats + 3, (unsigned long long)st_app);
-            atomicAdd(p.stats + 4, (unsigned long long)st_rcall);
-            atomicAdd(p.stats + 5, (unsigned long long)st_riter);
+            atomicAdd(p.stats + 4, (unsigned long long)st_fold);
             atomicAdd(p.stats + 8, (unsigned long long)st_twait);
-            atomicAdd(p.stats + 9, (unsigned long long)st_tproc);
             atomicAdd(p.stats + 10, (unsigned long long)(clock64() - st_t0));
             atomicAdd(p.stats + 11, 1ull);
-            atomicAdd(p.stats + 12, (unsigned long long)st_tref);
-            atomicAdd(p.stats + 13, (unsigned long long)(st_k1 - st_k0));
-            atomicAdd(p.stats + 14, (unsigned long long)(st_t0 - st_k1));
-            atomicAdd(p.stats + 2, (unsigned long long)(st_k0 - st_top));
+            atomicAdd(p.stats + 12, (unsigned long long)st_tfold);
         }
 #endif
 
-        // ---- finish.  All 256 epilogue threads meet here, also after an abort, so the decision is uniform.
-        asm volatile("bar.sync 1, 256;" ::: "memory");
+        // ---- finish.  All 512 epilogue threads meet at every barrier below, also after an abort.
+        auto epi_sync = [&]() { asm volatile("bar.sync 1, 512;" ::: "memory"); };
+        if (FILTER && S.overflow && row_live) atomicAdd(flagged, 1);
+        epi_sync();                                          // the candidate / zone / z areas are idle from here on
+        const bool aborted = *abort_flag != 0;
+
+        if (FILTER && !aborted) {
+            // ---- fallback: tokens whose zone overflowed are routed again, exactly, over this group's experts; the
+            // result replaces the token's list.  Rounds of kFallbackSlots tokens, one warp per token.
+            const int nflag = *flagged;
+            if (nflag > 0) {
+                float* fz = reinterpret_cast<float*>(ring_ptr);                          // [slot][RPAD] z
+                int* frange = reinterpret_cast<int*>(ring_ptr + kFallbackSlots * RPAD * 4);   // [slot][2]
+                float* fv = reinterpret_cast<float*>(frange + kFallbackSlots * 2);        // [slot][KCAP]
+                int* fi = reinterpret_cast<int*>(fv + kFallbackSlots * KCAP);
+                int* ticket = fi + kFallbackSlots * KCAP;
+                if (etid == 0) *ticket = 0;
+                epi_sync();
+                bool mine = S.overflow && row_live;
+                for (int done = 0; done < nflag; done += kFallbackSlots) {
+                    int slot = -1;
+                    if (mine) {
+                        const int t = atomicAdd(ticket, 1);
+                        if (t < done + kFallbackSlots) slot = t - done; else atomicSub(ticket, 1);
+                    }
+                    // the token's z: the high part comes from tensor memory, which only whole warps can read
+                    if (warp_live && __any_sync(kFullMask, slot >= 0)) {
+                        for (int c = 0; c < RPAD / 8; ++c) {
+                            uint32_t h4[4], l4[4];
+                            tmem_ld4(t_zop + c * 4, h4);
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(l4[0]), "=r"(l4[1]), "=r"(l4[2]), "=r"(l4[3])
+                                         : "r"(zlo_addr + c * (kEpiThreads * 16)) : "memory");
+                            tmem_ld_wait4(h4);
+                            if (slot >= 0) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    fz[slot * RPAD + c * 8 + 2 * e] = bf_lo(h4[e]) + bf_lo(l4[e]);
+                                    fz[slot * RPAD + c * 8 + 2 * e + 1] = bf_hi(h4[e]) + bf_hi(l4[e]);
+                                }
+                            }
+                        }
+                        if (slot >= 0) { frange[slot * 2] = e_lo; frange[slot * 2 + 1] = e_hi; }
+                    }
+                    epi_sync();
+                    const int nslots = min(kFallbackSlots, nflag - done);
+                    if (ew < nslots)
+                        exact_topk_warp<KCAP>(fz + ew * RPAD, p.R2, p.r, p.M, frange[ew * 2], frange[ew * 2 + 1],
+                                              fv + ew * KCAP, fi + ew * KCAP, lane);
+                    epi_sync();
+                    if (slot >= 0) {
+#pragma unroll
+                        for (int e = 0; e < KCAP; ++e) { L.v[e] = fv[slot * KCAP + e]; L.id[e] = fi[slot * KCAP + e]; }
+                        mine = false;
+                    }
+                    epi_sync();
+                }
+            }
+        }
+
+        if (es > 1 && !aborted) {
+            // ---- groups that share tokens: ranges 1.. park their lists in shared memory, range 0 merges them in
+            // ascending range order (equal logits keep the smaller id)
+            float* pv = reinterpret_cast<float*>(ring_ptr);                          // [tg][es-1][KCAP][128]
+            int* pi = reinterpret_cast<int*>(ring_ptr + kGroups * KCAP * 128 * 4);
+            float2* pmz = reinterpret_cast<float2*>(ring_ptr + 2 * kGroups * KCAP * 128 * 4);
+            if (warp_live && esi > 0) {
+                const int o = (tgi * (es - 1) + (esi - 1)) * KCAP * 128 + row_in_tg;
+#pragma unroll
+                for (int s = 0; s < KCAP; ++s) { pv[o + s * 128] = L.v[s]; pi[o + s * 128] = L.id[s]; }
+                pmz[(tgi * (es - 1) + (esi - 1)) * 128 + row_in_tg] = make_float2(m2, zsum);
+            }
+            epi_sync();
+            if (warp_live && esi == 0) {
+                for (int e = 1; e < es; ++e) {
+                    const int o = (tgi * (es - 1) + (e - 1)) * KCAP * 128 + row_in_tg;
+#pragma unroll
+                    for (int s = 0; s < KCAP; ++s) {
+                        const float x = pv[o + s * 128];
+                        if (x > L.tau()) L.insert(x, pi[o + s * 128]);
+                    }
+                    if (LSE) {
+                        const float2 mz = pmz[(tgi * (es - 1) + (e - 1)) * 128 + row_in_tg];
+                        if (mz.x > -INFINITY) {
+                            const float nm = fmaxf(m2, mz.x);
+                            zsum = zsum * ex2f(m2 - nm) + mz.y * ex2f(mz.x - nm);
+                            m2 = nm;
+                        }
+                    }
+                }
+            }
+            epi_sync();
+        }
+        const bool writer = row_live && esi == 0;            // one thread per token carries the result from here on
+
         // Expert histogram: when the M bins fit into the (now idle) ring, the CTA counts its tokens' ids in shared
         // memory and flushes only the non-zero bins with one global atomic each; otherwise straight to global memory
         // (with that many experts the bins hardly collide).  With few experts thousands of pairs hit each bin, and
         // same-address global atomics would serialise.
-        int* hist = (p.M * 4 <= kRingBytes) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
-        const int etid = threadIdx.x - 64;                   // 0..255 among the epilogue threads
+        int* hist = (p.M <= kRRing / 4) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
         auto hist_clear = [&]() {
             if (hist) {
-                for (int e = etid; e < p.M; e += kEpilogueThreads) hist[e] = 0;
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                for (int e = etid; e < p.M; e += kEpiThreads) hist[e] = 0;
+                epi_sync();
             }
         };
         auto hist_flush = [&]() {
             if (hist) {
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                for (int e = etid; e < p.M; e += kEpilogueThreads) {
+                epi_sync();
+                for (int e = etid; e < p.M; e += kEpiThreads) {
                     const int c = hist[e];
                     if (c) atomicAdd(p.out_counts + e, c);
                 }
             }
         };
-        if (*abort_flag == 0) {
+        if (!aborted) {
             if (p.msplit == 1) {
                 hist_clear();
-                if (row_live) write_token<KCAP>(p, row, L, m2, zsum, hist);
+                if (writer) write_token<KCAP>(p, row, L, m2, zsum, hist);
                 hist_flush();
             } else {
                 // park the partial list; the CTA that arrives last for this token block merges all of them
-                const int64_t slot = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit + split;
+                const int64_t slot = ((int64_t)blk * p.block_tokens + row_in_blk) * p.msplit + split;
+                if (writer) {
 #pragma unroll
-                for (int s = 0; s < KCAP; ++s) {
-                    p.part_val[slot * KCAP + s] = L.v[s];
-                    p.part_id[slot * KCAP + s] = L.id[s];
+                    for (int s = 0; s < KCAP; ++s) {
+                        p.part_val[slot * KCAP + s] = L.v[s];
+                        p.part_id[slot * KCAP + s] = L.id[s];
+                    }
+                    p.part_mz[slot] = make_float2(m2, zsum);
                 }
-                p.part_mz[slot] = make_float2(m2, zsum);
                 __threadfence();
-                asm volatile("bar.sync 1, 256;" ::: "memory");
-                if (threadIdx.x == 64) {
+                epi_sync();
+                if (etid == 0) {
                     const unsigned prev = atomicAdd(p.counters + blk, 1u);
                     *last_flag = (prev == (unsigned)p.msplit - 1u);
                 }
-                asm volatile("bar.sync 1, 256;" ::: "memory");
+                epi_sync();
                 if (*last_flag) {
                     __threadfence();
-                    const int64_t base = ((int64_t)blk * kBlockTokens + row_in_blk) * p.msplit;
+                    const int64_t base = ((int64_t)blk * p.block_tokens + row_in_blk) * p.msplit;
                     TopList<KCAP> G;
                     G.init();
                     float gm = -INFINITY, gz = 0.f;
-                    // A token's partial lists lie one after the other in scratch.  Each list's head (its four best
-                    // entries, which is all most lists contribute) is fetched with two 16-byte loads, and the next
-                    // list's head is requested before the current one is merged, so the L2 round trips overlap
-                    // instead of adding up; the tail of a list is read only if its fourth entry still got in.
-                    const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
-                    const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
-                    float4 hv = __ldcg(pv);
-                    int4 hi = __ldcg(pi);
-                    for (int sp = 0; sp < p.msplit; ++sp) {       // ascending expert ranges: ties keep the smaller id
-                        const float4 cv = hv;
-                        const int4 ci = hi;
-                        if (sp + 1 < p.msplit) {
-                            hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
-                            hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
-                        }
-                        // each partial list is sorted: stop at the first entry that does not get in
-                        bool more = cv.x > G.tau();
-                        if (more) G.insert(cv.x, ci.x);
-                        more = more && cv.y > G.tau();
-                        if (more) G.insert(cv.y, ci.y);
-                        more = more && cv.z > G.tau();
-                        if (more) G.insert(cv.z, ci.z);
-                        more = more && cv.w > G.tau();
-                        if (more) G.insert(cv.w, ci.w);
-                        for (int s = 4; s < KCAP && more; ++s) {
-                            const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
-                            const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
-                            more = x > G.tau();
-                            if (more) G.insert(x, j);
-                        }
-                        const float2 mz = __ldcg(p.part_mz + base + sp);
-                        if (LSE && mz.x > -INFINITY) {
-                            const float nm = fmaxf(gm, mz.x);
-                            gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
-                            gm = nm;
+                    if (writer) {
+                        // A token's partial lists lie one after the other in scratch.  Each list's head (its four best
+                        // entries, which is all most lists contribute) is fetched with two 16-byte loads, and the next
+                        // list's head is requested before the current one is merged, so the L2 round trips overlap;
+                        // the tail of a list is read only if its fourth entry still got in.
+                        const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
+                        const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
+                        float4 hv = __ldcg(pv);
+                        int4 hi = __ldcg(pi);
+                        for (int sp = 0; sp < p.msplit; ++sp) {       // ascending expert ranges: ties keep the smaller id
+                            const float4 cv = hv;
+                            const int4 ci = hi;
+                            if (sp + 1 < p.msplit) {
+                                hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
+                                hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
+                            }
+                            // each partial list is sorted: stop at the first entry that does not get in
+                            bool more = cv.x > G.tau();
+                            if (more) G.insert(cv.x, ci.x);
+                            more = more && cv.y > G.tau();
+                            if (more) G.insert(cv.y, ci.y);
+                            more = more && cv.z > G.tau();
+                            if (more) G.insert(cv.z, ci.z);
+                            more = more && cv.w > G.tau();
+                            if (more) G.insert(cv.w, ci.w);
+                            for (int s = 4; s < KCAP && more; ++s) {
+                                const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
+                                const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
+                                more = x > G.tau();
+                                if (more) G.insert(x, j);
+                            }
+                            const float2 mz = __ldcg(p.part_mz + base + sp);
+                            if (LSE && mz.x > -INFINITY) {
+                                const float nm = fmaxf(gm, mz.x);
+                                gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
+                                gm = nm;
+                            }
                         }
                     }
                     hist_clear();
-                    if (row_live) write_token<KCAP>(p, row, G, gm, gz, hist);
+                    if (writer) write_token<KCAP>(p, row, G, gm, gz, hist);
                     hist_flush();
-                    if (threadIdx.x == 64) p.counters[blk] = 0;   // ready for the next call
+                    if (etid == 0) p.counters[blk] = 0;      // ready for the next call
                 }
             }
         }
@@ -683,11 +894,6 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // ---- common exit: everyone arrives here, also after an abort
     tc_fence_before();
     __syncthreads();
-    STAT(if (threadIdx.x == 64 && p.stats) {
-        atomicAdd(p.stats + 6, (unsigned long long)(clock64() - st_top));      // CTA lifetime, clk
-        atomicMax(p.stats + 7, (unsigned long long)(clock64() - st_top));      // longest CTA
-        atomicAdd(p.stats + 15, 1ull);
-    })
     if (*abort_flag && threadIdx.x == 0) {
         // give bulk copies that may still be in flight time to land before shared memory is released
         for (int i = 0; i < 200; ++i) __nanosleep(1000);
@@ -695,109 +901,143 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------ preparation (filter mode)
+// For the filter: R2T[j][i] = R2[i][j] (bf16, [M][RPAD], ranks >= r zero), the largest Euclidean column norm of R2
+// (slightly inflated, so that rounding cannot make it too small), and out_counts cleared.  One CTA per 64 experts;
+// the CTA that finishes last reduces the per-CTA maxima (the arrival counter returns to zero for the next call).
+__global__ void __launch_bounds__(256)
+route_prepare_kernel(const __nv_bfloat16* __restrict__ R2, int r, int rpad, int M, __nv_bfloat16* __restrict__ r2t,
+                     float* __restrict__ partial, float* __restrict__ colnorm_max, unsigned* __restrict__ arrivals,
+                     int32_t* __restrict__ out_counts)
+{
+    __shared__ __nv_bfloat16 tile[64][64 + 8];      // [rank][expert], padded rows
+    __shared__ float red[64];
+    __shared__ int last;
+    const int j0 = blockIdx.x * 64;
+    const int tj = threadIdx.x & 63, ti = threadIdx.x >> 6;
+    for (int i = ti; i < rpad; i += 4) {
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (i < r && j0 + tj < M) v = R2[(int64_t)i * M + j0 + tj];
+        tile[i][tj] = v;
+    }
+    if (threadIdx.x < 64 && j0 + threadIdx.x < M) out_counts[j0 + threadIdx.x] = 0;
+    __syncthreads();
+    if (threadIdx.x < 64) {
+        float s = 0.f;
+        for (int i = 0; i < rpad; ++i) {
+            const float x = __bfloat162float(tile[i][threadIdx.x]);
+            s = fmaf(x, x, s);
+        }
+        red[threadIdx.x] = s;
+    }
+    // transposed rows: 16 bytes (8 ranks) per item
+    const int chunks = rpad / 8;
+    for (int item = threadIdx.x; item < 64 * chunks; item += 256) {
+        const int jj = item / chunks, c = item % chunks;
+        if (j0 + jj < M) {
+            uint32_t w[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+                w[e] = (uint32_t)__bfloat16_as_ushort(tile[c * 8 + 2 * e][jj]) |
+                       ((uint32_t)__bfloat16_as_ushort(tile[c * 8 + 2 * e + 1][jj]) << 16);
+            reinterpret_cast<uint4*>(r2t)[(size_t)(j0 + jj) * chunks + c] = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float m = 0.f;
+        for (int i = 0; i < 64; ++i) m = fmaxf(m, red[i]);
+        partial[blockIdx.x] = m;
+        __threadfence();
+        last = (atomicAdd(arrivals, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (last) {
+        __threadfence();
+        float m = 0.f;
+        for (int i = threadIdx.x; i < (int)gridDim.x; i += 256) m = fmaxf(m, __ldcg(partial + i));
+        __shared__ float red2[256];
+        red2[threadIdx.x] = m;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int i = 1; i < 256; ++i) m = fmaxf(m, red2[i]);
+            *colnorm_max = sqrtf(m) * 1.0001f;
+            *arrivals = 0;
+        }
     }
 }
 
 // ------------------------------------------------------------------------------------------------ host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using KernelFn = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const RouteParams);
 
-EncodeTiledFn encode_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// 2-D bf16 row-major tensor [rows][cols], box = box_cols x box_rows, 128-byte swizzle, zero fill out of bounds.
-struct MapKey {
-    const void* ptr;
-    int rows, cols, box_rows, box_cols;
-    bool operator==(const MapKey& o) const
-    {
-        return ptr == o.ptr && rows == o.rows && cols == o.cols && box_rows == o.box_rows && box_cols == o.box_cols;
-    }
-};
-constexpr int kMapCache = 128;
-MapKey g_keys[kMapCache];
-CUtensorMap g_maps[kMapCache];
-int g_map_count = 0, g_map_next = 0;
-
-}  // namespace
-
-int get_tensor_map(const void* ptr, int rows, int cols, int box_rows, int box_cols, CUtensorMap* out)
-{
-    const MapKey key{ptr, rows, cols, box_rows, box_cols};
-    for (int i = 0; i < g_map_count; ++i)
-        if (g_keys[i] == key) { *out = g_maps[i]; return MORE_OK; }
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return MORE_ERR_CUDA;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUtensorMap m;
-    CUresult res = fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    if (res != CUDA_SUCCESS) return MORE_ERR_CUDA;
-    const int slot = (g_map_count < kMapCache) ? g_map_count++ : (g_map_next++ % kMapCache);
-    g_keys[slot] = key;
-    g_maps[slot] = m;
-    *out = m;
-    return MORE_OK;
-}
-
-namespace {
-
-template <int RPAD, int KCAP, bool LSE, bool FULL>
-int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp, int ctas,
-               cudaStream_t st)
+// The instantiation for (RPAD, KCAP, MODE), with its shared-memory limit raised on the current device; null on failure.
+template <int RPAD, int KCAP, int MODE>
+KernelFn kernel_ready()
 {
     static unsigned long long configured = 0;   // one bit per device, per instantiation; guarded by the API mutex
-    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE, FULL>;
+    KernelFn kern = route_lowrank_kernel<RPAD, KCAP, MODE>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (!(configured >> (dev & 63) & 1ull)) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
-            return MORE_ERR_CUDA;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRSmem) != cudaSuccess)
+            return nullptr;
         configured |= 1ull << (dev & 63);
     }
-    kern<<<ctas, kThreads, kSmemBytes, st>>>(mx, m1, m2, kp);
-    count_launch(1);
-    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+    return kern;
 }
 
-template <int RPAD, int KCAP, bool FULL>
-int launch_lse(bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp,
-               int ctas, cudaStream_t st)
+template <int RPAD, int KCAP>
+KernelFn kernel_mode(int mode)
 {
-    return lse ? launch_one<RPAD, KCAP, true, FULL>(mx, m1, m2, kp, ctas, st)
-               : launch_one<RPAD, KCAP, false, FULL>(mx, m1, m2, kp, ctas, st);
+    switch (mode) {
+        case kModeExact: return kernel_ready<RPAD, KCAP, kModeExact>();
+        case kModeExactLse: return kernel_ready<RPAD, KCAP, kModeExactLse>();
+        default:
+            if constexpr (KCAP <= 16) return kernel_ready<RPAD, KCAP, kModeFilter>();
+            else return nullptr;
+    }
 }
 
-template <int RPAD, bool FULL = false>
-int launch_kcap(int k, bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2,
-                const KernelParams& kp, int ctas, cudaStream_t st)
+template <int RPAD>
+KernelFn kernel_kcap(int k, int mode)
 {
-    if (k <= 8) return launch_lse<RPAD, 8, FULL>(lse, mx, m1, m2, kp, ctas, st);
-#ifdef MORE_ONLY_K8
-    return MORE_ERR_SHAPE;
-#endif
-    if (k <= 16) return launch_lse<RPAD, 16, FULL>(lse, mx, m1, m2, kp, ctas, st);
-    return launch_lse<RPAD, 32, FULL>(lse, mx, m1, m2, kp, ctas, st);
+    if (k <= 8) return kernel_mode<RPAD, 8>(mode);
+    if (k <= 16) return kernel_mode<RPAD, 16>(mode);
+    return kernel_mode<RPAD, 32>(mode);
 }
 
 int kcap_of(int k) { return k <= 8 ? 8 : (k <= 16 ? 16 : 32); }
+int rpad_of(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct ScratchLayout {
+    size_t counters, part_val, part_id, part_mz, r2t, partial, total;
+};
+
+ScratchLayout scratch_layout(const RouteArgs& a, const Plan& p)
+{
+    ScratchLayout L{};
+    size_t off = 0;
+    if (p.msplit > 1) {
+        const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
+        const size_t slots = blocks * (size_t)p.block_tokens * (size_t)p.msplit;
+        const size_t kc = (size_t)kcap_of(a.k);
+        L.counters = off; off += align_up(blocks * 4, 256);
+        L.part_val = off; off += align_up(slots * kc * 4, 256);
+        L.part_id = off; off += align_up(slots * kc * 4, 256);
+        L.part_mz = off; off += align_up(slots * 8, 256);
+    }
+    if (p.filter) {
+        L.r2t = off; off += align_up((size_t)a.M * rpad_of(a.r) * 2, 256);
+        L.partial = off; off += align_up((size_t)((a.M + 63) / 64) * 4, 256);
+    }
+    L.total = off;
+    return L;
+}
 
 }  // namespace
 
@@ -806,62 +1046,87 @@ bool tcgen05_shape_ok(int T, int h, int r, int M, int k)
     return T >= 1 && h % 8 == 0 && M % 8 == 0 && r % 8 == 0 && r <= 64 && k <= 32;
 }
 
-size_t tcgen05_scratch_bytes(const RouteArgs& a, const Plan& p)
+size_t lowrank_scratch_bytes(const RouteArgs& a, const Plan& p) { return scratch_layout(a, p).total; }
+
+// Shared-memory plan of a launch: phase-1 stages from the bottom of the ring, R2 stages at its top.  Returns false if
+// the shape of the groups leaves no room (the planner never asks for such a shape).
+bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st1_bytes, int* nst2, int* st2_bytes,
+                       int* r2_off)
 {
-    if (p.msplit <= 1) return 0;
-    const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
-    const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
-    const size_t kc = (size_t)kcap_of(a.k);
-    return align_up(blocks * 4, 256) + align_up(slots * kc * 4, 256) * 2 + align_up(slots * 8, 256);
+    const int st2 = es * rpad * 128;
+    const int fixed = kCandBytes + (filter ? kZoneBytes + kEpiThreads * rpad * 2 : 0);
+    int n2 = (kRRing - fixed) / st2;
+    if (n2 > 8) n2 = 8;
+    const int st1 = tg * kXGroupBytes + kR1Bytes;
+    // phase 1 wants at least two stages below the R2 stages
+    while (n2 > 2 && kRRing - n2 * st2 < 2 * st1) --n2;
+    if (n2 < 2) return false;
+    const int off = (kRRing - n2 * st2) & ~1023;
+    int n1 = off / st1;
+    if (n1 > 4) n1 = 4;
+    if (n1 < 1) return false;
+    *nst1 = n1; *st1_bytes = st1; *nst2 = n2; *st2_bytes = st2; *r2_off = off;
+    return true;
 }
 
-int launch_tcgen05(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
+int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
 {
+    const int rpad = rpad_of(a.r);
+    RouteParams rp{};
+    if (!lowrank_smem_plan(rpad, p.tg, p.es, p.filter, &rp.nst1, &rp.st1_bytes, &rp.nst2, &rp.st2_bytes, &rp.r2_off))
+        return MORE_ERR_SHAPE;
     CUtensorMap mx, m1, m2;
-    const int x_rows = (!a.full && p.block_tokens <= 128) ? 128 : kBlockTokens;
-    int rc = get_tensor_map(a.X, a.T, a.h, x_rows, 64, &mx);
-    const int rpad = a.full ? 64 : ((a.r <= 16) ? 16 : (a.r <= 32 ? 32 : 64));
-    if (a.full) {
-        // standard router: R2 is W [h][M]; its k-tiles are 64 x 64 boxes like R1's
-        if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.h, a.M, 64, 64, &m2);
-        m1 = m2;
-    } else {
-        if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
-        if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.r, a.M, rpad, 64, &m2);
-    }
+    int rc = get_tensor_map(a.X, a.T, a.h, 128, 64, &mx);
+    if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
+    if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.r, a.M, rpad, 64, &m2);
     if (rc != MORE_OK) return rc;
 
-    KernelParams kp;
-    kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
-    kp.block_tokens = p.block_tokens;
-    kp.x_rows = x_rows;
-    kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
-    kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
-    kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
-    kp.status = ctx.status;
-    kp.stats = ctx.stats;
-    kp.counters = nullptr; kp.part_val = nullptr; kp.part_id = nullptr; kp.part_mz = nullptr;
+    rp.T = a.T; rp.h = a.h; rp.r = a.r; rp.M = a.M; rp.k = a.k; rp.gate_mode = a.gate_mode;
+    rp.msplit = p.msplit; rp.es = p.es; rp.tg = p.tg;
+    rp.block_tokens = p.block_tokens;
+    rp.blocks64 = (a.M + 63) / 64;
+    rp.out_idx = a.out_idx; rp.out_gate = a.out_gate; rp.out_counts = a.out_counts;
+    rp.out_topval = a.out_topval; rp.out_lse = a.out_lse;
+    rp.status = ctx.status;
+    rp.stats = ctx.stats;
+    rp.R2 = a.R2;
+    const ScratchLayout L = scratch_layout(a, p);
+    char* base = static_cast<char*>(scratch);
     if (p.msplit > 1) {
-        const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
-        const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
-        const size_t kc = (size_t)kcap_of(a.k);
-        char* base = static_cast<char*>(scratch);
-        kp.counters = reinterpret_cast<unsigned*>(base);
-        base += align_up(blocks * 4, 256);
-        kp.part_val = reinterpret_cast<float*>(base);
-        base += align_up(slots * kc * 4, 256);
-        kp.part_id = reinterpret_cast<int*>(base);
-        base += align_up(slots * kc * 4, 256);
-        kp.part_mz = reinterpret_cast<float2*>(base);
-        if (cudaMemsetAsync(kp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
+        rp.counters = reinterpret_cast<unsigned*>(base + L.counters);
+        rp.part_val = reinterpret_cast<float*>(base + L.part_val);
+        rp.part_id = reinterpret_cast<int*>(base + L.part_id);
+        rp.part_mz = reinterpret_cast<float2*>(base + L.part_mz);
     }
     const bool lse = (a.gate_mode == MORE_GATE_FULL_SOFTMAX) || (a.out_lse != nullptr);
-    if (a.full) return launch_kcap<64, true>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
-    switch (rpad) {
-        case 16: return launch_kcap<16>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
-        case 32: return launch_kcap<32>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
-        default: return launch_kcap<64>(a.k, lse, mx, m1, m2, kp, p.ctas, a.stream);
+    int mode = lse ? kModeExactLse : kModeExact;
+    if (p.filter) {
+        if (lse || a.k > 16) return MORE_ERR_SHAPE;
+        mode = kModeFilter;
     }
+    KernelFn kern = rpad == 16 ? kernel_kcap<16>(a.k, mode) : (rpad == 32 ? kernel_kcap<32>(a.k, mode) : kernel_kcap<64>(a.k, mode));
+    if (!kern) return MORE_ERR_CUDA;
+    // every host-side step that can fail is behind us: only now is anything enqueued and the first output touched
+    if (p.msplit > 1) {
+        const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
+        if (cudaMemsetAsync(rp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
+    }
+    if (p.filter) {
+        __nv_bfloat16* r2t = reinterpret_cast<__nv_bfloat16*>(base + L.r2t);
+        rp.r2t = r2t;
+        rp.colnorm_max = ctx.colnorm_max;
+        // the preparation kernel also clears out_counts
+        route_prepare_kernel<<<(a.M + 63) / 64, 256, 0, a.stream>>>(a.R2, a.r, rpad, a.M, r2t,
+                                                                   reinterpret_cast<float*>(base + L.partial),
+                                                                   ctx.colnorm_max, ctx.prep_arrivals, a.out_counts);
+        count_launch(1);
+        if (cudaGetLastError() != cudaSuccess) return MORE_ERR_CUDA;
+    } else if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) {
+        return MORE_ERR_CUDA;
+    }
+    kern<<<p.ctas, kRThreads, kRSmem, a.stream>>>(mx, m1, m2, rp);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
 }
 
 }  // namespace more

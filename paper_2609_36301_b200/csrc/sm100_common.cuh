@@ -4,6 +4,8 @@
 
 #include <cuda.h>   // CUtensorMap and the driver entry-point typedef only; libcuda is resolved at run time
 #include <cuda_runtime.h>
+#include <limits.h>
+#include <math.h>
 #include <stdint.h>
 
 #include "more_internal.h"
@@ -211,6 +213,70 @@ __device__ __forceinline__ float ex2f(float x)
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+
+// 4 consecutive 32-bit columns of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t (&u)[4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(u[0]), "=r"(u[1]), "=r"(u[2]), "=r"(u[3])
+                 : "r"(taddr)
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait4(uint32_t (&u)[4])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;" : "+r"(u[0]), "+r"(u[1]), "+r"(u[2]), "+r"(u[3]) : : "memory");
+}
+
+// One arrival for the whole (converged) warp: the lanes' own tensor-memory accesses have completed (wait::ld /
+// wait::st are warp-wide), the warp synchronises, lane 0 arrives.  The barrier counts warps, not threads.
+__device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
+{
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar);
+}
+
+// ---------------------------------------------------------------------------------------------- running top-k
+// Sorted (value, id) list of one token, held in registers.
+template <int KCAP>
+struct TopList {
+    float v[KCAP];
+    int id[KCAP];
+    __device__ __forceinline__ void init()
+    {
+#pragma unroll
+        for (int s = 0; s < KCAP; ++s) { v[s] = -INFINITY; id[s] = INT_MAX; }
+    }
+    __device__ __forceinline__ float tau() const { return v[KCAP - 1]; }
+    // Insert (x, j) with x > tau().  Equal values keep the earlier (smaller-id) entry ahead.
+    __device__ __forceinline__ void insert(float x, int j)
+    {
+#pragma unroll
+        for (int s = KCAP - 1; s > 0; --s) {
+            const bool above_prev = x > v[s - 1];
+            const bool above_this = x > v[s];
+            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
+            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
+        }
+        const bool top = x > v[0];
+        v[0] = top ? x : v[0];
+        id[0] = top ? j : id[0];
+    }
+    // Insert with the full order (value descending, id ascending): for merging lists whose ids interleave.
+    __device__ __forceinline__ void insert_ordered(float x, int j)
+    {
+        auto ahead = [&](int s) { return x > v[s] || (x == v[s] && j < id[s]); };
+#pragma unroll
+        for (int s = KCAP - 1; s > 0; --s) {
+            const bool above_prev = ahead(s - 1);
+            const bool above_this = ahead(s);
+            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
+            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
+        }
+        const bool top = ahead(0);
+        v[0] = top ? x : v[0];
+        id[0] = top ? j : id[0];
+    }
+};
 
 // ------------------------------------------------------------------------------------------- UMMA descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
