@@ -34,7 +34,7 @@ struct DeviceCtx {
     unsigned long long* stats = nullptr;   // 16 diagnostic counters, next to the status word
     void* staging = nullptr;      // device staging of more_route_host
     size_t staging_bytes = 0;
-    float* colnorm_max = nullptr;       // device float: largest column norm of R2, written by the filter's preparation
+    float* colnorm = nullptr;           // device float[2]: column-norm maxima written by the filter's preparation
     unsigned* prep_arrivals = nullptr;  // device counter of that kernel (returns to zero after every launch)
 };
 

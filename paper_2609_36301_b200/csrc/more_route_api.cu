@@ -32,8 +32,8 @@ int get_ctx(DeviceCtx** out)
         if (cudaMalloc(&blk, 256) != cudaSuccess) return MORE_ERR_CUDA;
         if (cudaMemset(blk, 0, 256) != cudaSuccess) return MORE_ERR_CUDA;
         c.status = static_cast<int*>(blk);
-        c.colnorm_max = reinterpret_cast<float*>(static_cast<char*>(blk) + 64);
-        c.prep_arrivals = reinterpret_cast<unsigned*>(static_cast<char*>(blk) + 68);
+        c.colnorm = reinterpret_cast<float*>(static_cast<char*>(blk) + 64);
+        c.prep_arrivals = reinterpret_cast<unsigned*>(static_cast<char*>(blk) + 72);
         c.stats = reinterpret_cast<unsigned long long*>(static_cast<char*>(blk) + 128);
         c.dev = dev;
     }

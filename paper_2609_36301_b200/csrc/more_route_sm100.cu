@@ -2,9 +2,13 @@
 // and the per-expert counts fused in).  One CTA per SM, 18 warps:
 //
 //   warp 0       TMA producer: X and R1 k-tiles for phase 1, R2 blocks of 64 experts for phase 2.
-//   warp 1       tensor-memory allocation and tcgen05.mma issue (the warp stays converged, one elected lane issues).
+//   warp 1       tensor-memory allocation and the tcgen05.mma issue of phase 1.
 //   warps 2..17  epilogue: four groups of four warps.  A group owns 128 tensor-memory lanes = 128 tokens and one
-//                contiguous range of experts; a thread owns one token of its group.
+//                contiguous range of experts; a thread owns one token of its group.  The groups feed themselves in
+//                phase 2: whichever warp of a group is the last to have read an accumulator buffer out issues, there
+//                and then, the MMAs that refill it (the warp stays converged, one elected lane issues).  A separate
+//                issuing warp adds its own wake-up and a chain of slow synchronising instructions to every hand-over,
+//                and measured several hundred clocks per 32-column buffer.
 //
 // A CTA routes `block_tokens` (<= 512) tokens.  Its four groups are laid out as tg token groups x es expert ranges
 // (tg * es <= 4): with many tokens per SM every group takes different tokens and sweeps all of the CTA's experts; with
@@ -13,20 +17,29 @@
 // expert axis (partial lists parked in global scratch, merged by the CTA that finishes last).
 //
 //   phase 1  z = X_blk R1            128 x 64 X tiles and 64 x 64 R1 tiles by TMA, tcgen05.mma into fp32 accumulators.
-//   narrow   z -> bf16 operand       each group writes z into its own tensor-memory columns as the A operand of
-//                                    phase 2 (tcgen05.st): bf16 high part + bf16 low part in the exact modes, the high
-//                                    part alone in filter mode.
+//   narrow   z -> 16-bit operand     each group writes z into its own tensor-memory columns as the A operand of
+//                                    phase 2 (tcgen05.st): bf16 high part + bf16 low part in the exact modes; in
+//                                    filter mode z scaled by a power of two and rounded to fp16, nothing else.
 //   phase 2  y = z R2[:, 32 experts] N = 32 MMAs with A from tensor memory fill a ring of 32-column accumulators per
-//                                    group (three, or two when the operand needs 64 columns); the epilogue warps drain
-//                                    them 16 columns at a time and hand each buffer back as soon as it is in registers,
-//                                    so the MMAs run up to a ring ahead of the slowest warp of a group.
+//                                    group (three, or two when the operand needs 64 columns); a warp copies a buffer
+//                                    into registers, counts itself out of it, and the last one refills it, so the
+//                                    MMAs run up to a ring ahead of the slowest warp of a group.  Every range is swept
+//                                    for the same number of steps; what lies beyond a range's end is masked.
 //   select   running top-k           sorted list in registers fed through a per-token candidate buffer in shared
 //                                    memory (Selector).
 //   finish   gates, ids, counts.
 //
-// Filter mode (top-k-softmax gate, no log-sum-exp wanted).  The second contraction runs on the high part of z only,
-// which halves its tensor work and frees tensor memory for the ring, but perturbs each logit by up to
-// E = |z - hi(z)|_2 * max_j |R2[:, j]|_2 (Cauchy-Schwarz; about 1e-2).  The sweep therefore keeps, besides the running
+// Filter mode (top-k-softmax gate, no log-sum-exp wanted).  The second contraction runs on one 16-bit rounding of z
+// only, which halves its tensor work and frees tensor memory for the ring, but perturbs each logit by up to
+// E = |z - hi(z)|_2 * max_j |R2[:, j]|_2 (Cauchy-Schwarz).  hi(z) is fp16, not bf16: three more mantissa bits make E
+// ~2e-3 of the logits' spread instead of ~2e-2.  Both operands of a kind::f16 MMA must then be fp16 (a bf16 B with an
+// fp16 A is an illegal instruction on this part), so the preparation kernel also writes an fp16 copy of R2, which the
+// sweep reads instead of R2; bf16 values convert exactly unless they leave fp16's exponent range, and the Euclidean
+// norm of each column's conversion error enters the bound (it is zero or ~1e-8 for sane weights, and infinite --
+// sending every token to the fallback -- if a weight overflows fp16).  Every token's z is first scaled by a power of
+// two that puts its largest component near 2^13, so z neither overflows nor goes subnormal whatever the scale of the
+// inputs (the approximate logits of a token are all scaled alike, which selection does not see).  The sweep keeps,
+// besides the running
 // top-k of the approximate logits, every expert within W = 2E below the k-th of them (the "zone": any expert of the
 // true top-k lies there), and the survivors' logits are then recomputed in fp32 from the full z and the expert's
 // column (a row of the transposed copy of R2 the preparation kernel writes), which decides the final top-k, order
@@ -36,6 +49,10 @@
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device status
 // word, raises the CTA's abort flag and all roles fall through to the common exit (tensor memory is freed there).
 #include "sm100_common.cuh"
+
+#include <cuda_fp16.h>
+
+#include <type_traits>
 
 #ifdef MORE_STATS
 #define STAT(...) __VA_ARGS__
@@ -49,12 +66,16 @@ namespace {
 
 constexpr int kGroups = 4;                         // 128-token groups per CTA
 constexpr int kEpiThreads = 128 * kGroups;
-constexpr int kRThreads = 64 + kEpiThreads;        // warps 0, 1 + 16 epilogue warps
+constexpr int kFirstEpiWarp = 2;
+constexpr int kRThreads = 32 * kFirstEpiWarp + kEpiThreads;   // TMA warp, phase-1 MMA warp, 16 epilogue warps
 constexpr int kRRing = 208 * 1024;                 // shared-memory working area
 constexpr int kRSmem = kRRing + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
 constexpr int kGroupCols = 128;                    // tensor-memory columns per group
 constexpr int kBufCols = 32;                       // one accumulator buffer of the ring
-constexpr int kCandCap = 8;                        // candidate slots per token
+#ifndef MORE_CAND_CAP
+#define MORE_CAND_CAP 12
+#endif
+constexpr int kCandCap = MORE_CAND_CAP;            // candidate slots per token
 constexpr int kCandValStride = kEpiThreads * 16;   // bytes between successive value slots of one thread
 constexpr int kCandColStride = kEpiThreads * 4;    // ... and between its column slots
 constexpr int kCandValBytes = kCandCap * kCandValStride;
@@ -90,10 +111,12 @@ struct RouteParams {
     float* part_val;
     int* part_id;
     float2* part_mz;
-    // filter mode: transposed copy of R2 ([M][RPAD] bf16, columns >= r zero) and the largest column norm of R2
+    // filter mode: transposed copy of R2 ([M][RPAD] bf16, columns >= r zero); colnorm[0] = largest column norm of R2,
+    // colnorm[1] = largest column norm of the error of its fp16 copy
     const __nv_bfloat16* r2t;
-    const float* colnorm_max;
+    const float* colnorm;
     const __nv_bfloat16* R2;     // for the fallback sweep
+    uint4* zlo;                  // filter: the low halves of z, [CTA][rank / 8][512 threads] x 16 B
 };
 
 // ---------------------------------------------------------------------------------------- shared-memory access
@@ -142,7 +165,7 @@ struct Selector {
         W = w;
         base = ptr = first_val_slot;
         cbase = cptr = first_col_slot;
-        warn = first_val_slot + (kCandCap - 4) * kCandValStride;
+        warn = first_val_slot + (kCandCap - 8) * kCandValStride;      // a 32-column buffer appends at most 8 entries
         zbase = zptr = first_zone_slot;
         overflow = false;
     }
@@ -174,6 +197,9 @@ struct Selector {
     // (rising) limit any more moves on to its next entries.  The rounds end when no token has anything left.
     __device__ __forceinline__ void fold()
     {
+#ifdef MORE_EXP_NOFOLD
+        ptr = base; cptr = cbase; thr = 3.2f; return;      // timing experiment: what the scan alone costs
+#endif
         uint32_t a = base, c = cbase;
         float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
         int col = 0;
@@ -316,7 +342,6 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kRingCol0 = (kZopCols <= 32) ? 32 : 64;            // first column of the accumulator ring
     constexpr int NBUF = (kGroupCols - kRingCol0) / kBufCols;        // 3 or 2
     constexpr int kR2BlockBytes = RPAD * 128;                        // RPAD rows x 64 experts
-    constexpr int kZloOff = kCandBytes + kZoneBytes;                 // filter: low part of z, 16 B per (8 ranks, thread)
     using Sel = Selector<KCAP, FILTER>;
 
     extern __shared__ uint8_t smem_raw[];
@@ -325,13 +350,16 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint8_t* ring_ptr = smem_raw + (ring - raw);
     uint8_t* ctl = ring_ptr + kRRing;                        // control block
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
-    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + 4, B_ZACC = B_EMPTY1 + 4, B_ZOP = B_ZACC + 1,
-                  B_FULL2 = B_ZOP + kGroups, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8,
-                  B_ACCE = B_ACCF + kGroups * 3, B_COUNT = B_ACCE + kGroups * 3;
+    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + 4, B_ZACC = B_EMPTY1 + 4, B_FULL2 = B_ZACC + 1,
+                  B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_COUNT = B_ACCF + kGroups * 3;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
     int* flagged = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 12);      // tokens that need the fallback sweep
+    int* part_tab = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 16);    // [es]: first 64-expert block of every range
+    int* zop_done = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 32);    // [tg]: warps that have written their operand
+    int* released = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 48);    // [group][slot]: warps that have read a buffer out
+    STAT(long long* issue_clk = reinterpret_cast<long long*>(ctl + B_COUNT * 8 + 96);)   // [group][slot]: when the refill was issued
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -343,24 +371,24 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const int es = p.es;
     const int ngroups = tg_live * es;
     const int nparts = p.msplit * es;
-    // 64-expert blocks of expert range `esi` of this CTA: an even share of ceil(M / 64) blocks
-    auto part_lo = [&](int esi) { return (int)(((long long)p.blocks64 * (split * es + esi)) / nparts); };
-    auto part_hi = [&](int esi) { return (int)(((long long)p.blocks64 * (split * es + esi + 1)) / nparts); };
+    // 64-expert blocks of expert range `esi` of this CTA: an even share of ceil(M / 64) blocks.  The shares differ by
+    // at most one block; every range is swept for nsteps blocks all the same, and whatever that reads beyond the
+    // range's own end (the next range's first block, or zero fill past M) is masked in the epilogue.
+    auto part_lo = [&](int esi) { return part_tab[esi]; };
     auto live_warps = [&](int tgi) { return min(4, (live_tokens - tgi * 128 + 31) >> 5); };
     const int ktiles1 = (p.h + 63) / 64;
-    int nsteps_max = 0;
-    for (int e = 0; e < es; ++e) nsteps_max = max(nsteps_max, part_hi(e) - part_lo(e));
+    const int nsteps = (p.blocks64 + nparts - 1) / nparts;
+    const int nst2_mask = p.nst2 - 1;                        // nst2 is a power of two
+    const int nst2_shift = 31 - __clz(p.nst2);
 
     if (threadIdx.x == 0) {
+        for (int e = 0; e < es; ++e) part_tab[e] = (int)(((long long)p.blocks64 * (split * es + e)) / nparts);
         for (int i = 0; i < 4; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
         mbar_init(bar(B_ZACC), 1);
-        for (int t = 0; t < kGroups; ++t) mbar_init(bar(B_ZOP + t), t < tg_live ? es * live_warps(t) : 1);
-        for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
-        for (int g = 0; g < kGroups; ++g)
-            for (int s = 0; s < 3; ++s) {
-                mbar_init(bar(B_ACCF + g * 3 + s), 1);
-                mbar_init(bar(B_ACCE + g * 3 + s), g < ngroups ? live_warps(g / es) : 1);
-            }
+        // a stage is free again when both 32-expert halves of every group's step have been multiplied
+        for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 2 * ngroups); }
+        for (int i = 0; i < kGroups * 3; ++i) { mbar_init(bar(B_ACCF + i), 1); released[i] = 0; }
+        for (int t = 0; t < kGroups; ++t) zop_done[t] = 0;
         *abort_flag = 0;
         *last_flag = 0;
         *flagged = 0;
@@ -394,86 +422,47 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 tma_load_2d(dst + p.tg * kXGroupBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
             }
             // the R2 stages lie beyond the phase-1 stages, so the first blocks of R2 arrive while phase 1 still runs
-            for (int it = 0; it < nsteps_max && ok; ++it) {
-                const int s = it % p.nst2;
-                if (it >= p.nst2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it / p.nst2) - 1) & 1, abort_flag, p.status);
+            for (int it = 0; it < nsteps && ok; ++it) {
+                const int s = it & nst2_mask;
+                if (it >= p.nst2) ok = mbar_wait(bar(B_EMPTY2 + s), ((it >> nst2_shift) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                int nb = 0;
-                for (int e = 0; e < es; ++e) nb += (it < part_hi(e) - part_lo(e));
-                mbar_expect_tx(bar(B_FULL2 + s), nb * kR2BlockBytes);
+                mbar_expect_tx(bar(B_FULL2 + s), es * kR2BlockBytes);
                 for (int e = 0; e < es; ++e)
-                    if (it < part_hi(e) - part_lo(e))
-                        tma_load_2d(r2ring + s * p.st2_bytes + e * kR2BlockBytes, &map_r2, bar(B_FULL2 + s),
-                                    (part_lo(e) + it) * 64, 0);
+                    tma_load_2d(r2ring + s * p.st2_bytes + e * kR2BlockBytes, &map_r2, bar(B_FULL2 + s),
+                                (part_lo(e) + it) * 64, 0);
             }
         }
     } else if (warp == 1) {
-        // ======================================================================================= MMA issuer
-        // The whole warp runs this code converged; one elected lane issues each tcgen05 instruction.
+        // ================================================================================== phase-1 MMA issuer
+        // The whole warp runs this code converged; one elected lane issues each tcgen05 instruction.  z of token group
+        // t accumulates in the ring columns of the group's first expert range.  Descriptor words of stage 0: K-major X
+        // tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address.
         bool ok = true;
         constexpr uint32_t idesc1 = umma_idesc(RPAD);
-        constexpr uint32_t idesc2 = umma_idesc(kBufCols);
-        {
-            // descriptor words of stage 0: K-major X tile (A), MN-major R1 tile (B); +2 per 32 bytes of start address
-            const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + p.tg * kXGroupBytes, 8192, 1024);
-            const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
-            for (int kt = 0; kt < ktiles1 && ok; ++kt) {
-                const int s = kt % p.nst1;
-                ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / p.nst1) & 1, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                const uint32_t x_lo = x_lo0 + s * (p.st1_bytes >> 4), r_lo = r_lo0 + s * (p.st1_bytes >> 4);
-                for (int t = 0; t < tg_live; ++t) {
-                    // z of token group t accumulates in the ring columns of its first group
-                    const uint32_t d = tmem_base + (t * es) * kGroupCols + kRingCol0;
+        const uint64_t xd = umma_desc_sw128(ring, 16, 1024), rd = umma_desc_sw128(ring + p.tg * kXGroupBytes, 8192, 1024);
+        const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), r_lo0 = (uint32_t)rd, r_hi = (uint32_t)(rd >> 32);
+        for (int kt = 0; kt < ktiles1 && ok; ++kt) {
+            const int s = kt % p.nst1;
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (kt / p.nst1) & 1, abort_flag, p.status));
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t x_lo = x_lo0 + s * (p.st1_bytes >> 4), r_lo = r_lo0 + s * (p.st1_bytes >> 4);
+            for (int t = 0; t < tg_live; ++t) {
+                const uint32_t d = tmem_base + (t * es) * kGroupCols + kRingCol0;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
-                        tc_mma_bf16_ss_elect(d, x_lo + t * (kXGroupBytes >> 4) + kk * 2, x_hi, r_lo + kk * (2048 >> 4),
-                                             r_hi, idesc1, (kt | kk) != 0);
-                }
-                tc_commit_elect(bar(B_EMPTY1 + s));
+                for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
+                    tc_mma_bf16_ss_elect(d, x_lo + t * (kXGroupBytes >> 4) + kk * 2, x_hi, r_lo + kk * (2048 >> 4),
+                                         r_hi, idesc1, (kt | kk) != 0);
             }
+            tc_commit_elect(bar(B_EMPTY1 + s));
         }
         if (ok) tc_commit_elect(bar(B_ZACC));
-        // every group has written its operand (and, where groups share tokens, read the shared z) before phase 2
-        for (int t = 0; t < tg_live; ++t) ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ZOP + t), 0, abort_flag, p.status));
-        tc_fence_after();
-        const uint64_t bd0 = umma_desc_sw128(r2ring, 8192, 1024);
-        const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
-        for (int it = 0; it < nsteps_max && ok; ++it) {
-            const int s = it % p.nst2;
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL2 + s), (it / p.nst2) & 1, abort_flag, p.status));
-            if (!ok) break;
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                const int n = it * 2 + half;                         // the groups' n-th 32-expert buffer
-                const int slot = n % NBUF;
-                const uint32_t use = (uint32_t)(n / NBUF);
-                for (int g = 0; g < ngroups && ok; ++g) {
-                    const int esi = g % es;
-                    if (it >= part_hi(esi) - part_lo(esi)) continue;
-                    // the slot is free once the group's warps have read its previous contents out
-                    if (use > 0) ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCE + g * 3 + slot), (use - 1) & 1, abort_flag, p.status));
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t d = tmem_base + g * kGroupCols + kRingCol0 + slot * kBufCols;
-                    const uint32_t a0 = tmem_base + g * kGroupCols;
-                    const uint32_t b_lo = b_lo0 + ((s * p.st2_bytes + esi * kR2BlockBytes) >> 4) + half * (64 >> 4);
-#pragma unroll
-                    for (int j = 0; j < kMmasPerBuf; ++j)       // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
-                        tc_mma_bf16_ts_elect(d, a0 + j * 8, b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
-                    tc_commit_elect(bar(B_ACCF + g * 3 + slot));
-                }
-            }
-            if (!ok) break;
-            tc_commit_elect(bar(B_EMPTY2 + s));
-        }
     } else {
         // ========================================================================================= epilogue
-        const int ew = warp - 2;
+        const int ew = warp - kFirstEpiWarp;
         const int g = ew >> 2;                               // group
         const int q = warp & 3;                              // TMEM lane quarter this warp may access
-        const int etid = threadIdx.x - 64;                   // 0..511 among the epilogue threads
+        const int etid = threadIdx.x - 32 * kFirstEpiWarp;   // 0..511 among the epilogue threads
         const int tgi = g / es, esi = g % es;
         const int row_in_tg = q * 32 + lane;
         const int row_in_blk = tgi * 128 + row_in_tg;
@@ -484,10 +473,33 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const uint32_t t_zacc = t_lanes + (tgi * es) * kGroupCols + kRingCol0;       // the token group's z (fp32)
         const uint32_t t_zop = t_lanes + g * kGroupCols;                              // this group's A operand
         const uint32_t t_ring = t_zop + kRingCol0;
-        const uint32_t zlo_addr = ring + kZloOff + etid * 16;
+        // filter: low half of this thread's z, 16 B per 8 ranks, in global scratch (read back once, for rescoring)
+        uint4* zlo = FILTER ? p.zlo + (size_t)blockIdx.x * (RPAD / 8) * kEpiThreads + etid : nullptr;
         const int e_lo = part_lo(esi) * 64;
-        const int e_hi = min(part_hi(esi) * 64, p.M);
-        const int nb = warp_live ? 2 * (part_hi(esi) - part_lo(esi)) : 0;             // 32-expert buffers to drain
+        // this range ends where the next one begins (the ranges of a CTA are consecutive shares of all parts)
+        const int e_hi = min((int)(((long long)p.blocks64 * (split * es + esi + 1)) / nparts) * 64, p.M);
+        const int nb = warp_live ? 2 * nsteps : 0;                                    // 32-expert buffers to drain
+        const int lw = live_warps(tgi);                                               // warps of this group with tokens
+
+        // ---- refill of the ring.  Buffer m of the group = 32-expert half (m & 1) of step m >> 1, in ring slot m % NBUF.
+        // Called by one whole warp, converged; an elected lane issues.  Both commits follow the MMAs of this buffer:
+        // one tells the group that the buffer is full, the other counts towards releasing the R2 stage.
+        constexpr uint32_t idesc2 = FILTER ? umma_idesc_f16(kBufCols) : umma_idesc(kBufCols);
+        const uint64_t bd0 = umma_desc_sw128(r2ring + esi * kR2BlockBytes, 8192, 1024);
+        const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+        auto issue_buffer = [&](int grp, uint32_t b_lo_grp, int m, int slot) -> bool {
+            const int it = m >> 1;
+            const int st = it & nst2_mask;
+            if (!mbar_wait(bar(B_FULL2 + st), (it >> nst2_shift) & 1, abort_flag, p.status)) return false;
+            tc_fence_after();
+            const uint32_t t_grp = tmem_base + grp * kGroupCols;
+            tc_mma_buffer_ts<kMmasPerBuf, kKSteps>(t_grp + kRingCol0 + slot * kBufCols, t_grp,
+                                                   b_lo_grp + st * (p.st2_bytes >> 4) + (m & 1) * (64 >> 4), b_hi, idesc2);
+            tc_commit_elect(bar(B_ACCF + grp * 3 + slot));
+            tc_commit_elect(bar(B_EMPTY2 + st));
+            STAT(if (lane == 0) issue_clk[grp * 3 + slot] = clock64();)
+            return true;
+        };
 
         float zone_w = 0.f;
         bool ok = true;
@@ -495,10 +507,27 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             ok = mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
             ok = __all_sync(kFullMask, ok);
         }
+        float zscale = 1.f;                                  // filter: z = (hi + lo) * zscale
         if (warp_live && ok) {
-            // ---- narrow z to bf16 and store it to tensor memory as the A operand of phase 2
+            // ---- narrow z and store it to tensor memory as the A operand of phase 2
             tc_fence_after();
-            float lo2 = 0.f, z2 = 0.f;
+            float lo2 = 0.f, z2 = 0.f, down = 1.f;
+            if (FILTER) {
+                // power of two that brings the token's largest |z| into [2^13, 2^14)
+                float zmax = 0.f;
+#pragma unroll
+                for (int c = 0; c < RPAD / 16; ++c) {
+                    float z[16];
+                    tmem_ld16(t_zacc + c * 16, z);
+                    tmem_ld_wait16(z);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) zmax = fmaxf(zmax, fabsf(z[e]));
+                }
+                int ex = (int)((__float_as_uint(zmax) >> 23) & 0xffu) - 127;      // floor(log2 zmax) for normal zmax
+                ex = (zmax > 0.f && zmax < INFINITY) ? max(-100, min(100, ex - 13)) : 0;
+                zscale = __uint_as_float((uint32_t)(127 + ex) << 23);
+                down = __uint_as_float((uint32_t)(127 - ex) << 23);
+            }
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
@@ -507,59 +536,79 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
-                    const float d0 = z[2 * e] - __bfloat162float(h0), d1 = z[2 * e + 1] - __bfloat162float(h1);
-                    const __nv_bfloat16 l0 = __float2bfloat16_rn(d0), l1 = __float2bfloat16_rn(d1);
-                    hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
                     if (FILTER) {
-                        // the part of z the approximate logits do not see, and z itself (hi + lo, as it is rescored)
+                        const float z0 = z[2 * e] * down, z1 = z[2 * e + 1] * down;
+                        const __half2 h = __floats2half2_rn(z0, z1);
+                        const float2 hf = __half22float2(h);
+                        const float d0 = z0 - hf.x, d1 = z1 - hf.y;
+                        const __half2 l = __floats2half2_rn(d0, d1);
+                        hi[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        lo[e] = *reinterpret_cast<const uint32_t*>(&l);
+                        // the part of z the approximate logits do not see, and the size of z itself
                         lo2 = fmaf(d0, d0, lo2);
                         lo2 = fmaf(d1, d1, lo2);
-                        z2 = fmaf(z[2 * e], z[2 * e], z2);
-                        z2 = fmaf(z[2 * e + 1], z[2 * e + 1], z2);
+                        z2 = fmaf(z0, z0, z2);
+                        z2 = fmaf(z1, z1, z2);
+                    } else {
+                        const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
+                        const float d0 = z[2 * e] - __bfloat162float(h0), d1 = z[2 * e + 1] - __bfloat162float(h1);
+                        const __nv_bfloat16 l0 = __float2bfloat16_rn(d0), l1 = __float2bfloat16_rn(d1);
+                        hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                        lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
                     }
                 }
                 tmem_st8(t_zop + c * 8, hi);
                 if (FILTER) {
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zlo_addr + (2 * c) * (kEpiThreads * 16)),
-                                 "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zlo_addr + (2 * c + 1) * (kEpiThreads * 16)),
-                                 "r"(lo[4]), "r"(lo[5]), "r"(lo[6]), "r"(lo[7]) : "memory");
+                    zlo[(2 * c) * kEpiThreads] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    zlo[(2 * c + 1) * kEpiThreads] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
                 } else {
                     tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
                 }
             }
             tmem_st_wait();
             tc_fence_before();
-            warp_arrive(bar(B_ZOP + tgi), lane);
+            // The last warp of the token group to get here (all expert ranges of the group counted: they read the
+            // same z, which the first range's ring is about to overwrite) starts phase 2 for every one of them.
+            __syncwarp();
+            int prior = 0;
+            if (lane == 0)
+                asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], 1;"
+                             : "=r"(prior) : "r"(smem_u32(zop_done + tgi)) : "memory");
+            prior = __shfl_sync(kFullMask, prior, 0);
+            if (prior == es * lw - 1) {
+                tc_fence_after();
+                for (int e = 0; e < es && ok; ++e)
+                    for (int m = 0; m < NBUF && m < nb && ok; ++m)
+                        ok = issue_buffer(tgi * es + e, b_lo0 + ((e - esi) * kR2BlockBytes >> 4), m, m);
+            }
+            ok = __all_sync(kFullMask, ok);
             if (FILTER) {
-                // |approximate - fp32 logit| <= |z - hi|_2 |R2_j|_2 (the missing low part) + accumulation rounding of
-                // the two evaluations (bounded by 2^-18 |z|_2 |R2_j|_2, a generous multiple of fp32 epsilon).
-                const float cn = __ldg(p.colnorm_max);
-                const float e_bound = sqrtf(lo2) * cn * 1.001f + sqrtf(z2) * cn * 3.8147e-6f;
-                zone_w = 2.f * e_bound * 1.001f + 1e-30f;
+                // |approximate - fp32 logit| (both in the scaled units of this token) <= |z - hi|_2 |R2_j|_2 for the
+                // part of z the sweep does not see, + |z|_2 |R2_j - fp16(R2_j)|_2 for what the fp16 copy of R2 lost,
+                // + the accumulation rounding of the two evaluations, bounded by 2^-18 |z|_2 |R2_j|_2 (a generous
+                // multiple of fp32 epsilon).
+                const float cn = __ldg(p.colnorm), cerr = __ldg(p.colnorm + 1);
+                const float e_bound = sqrtf(lo2) * cn * 1.001f + sqrtf(z2) * (cn * 3.8147e-6f + cerr * 1.001f);
+                zone_w = (e_bound == e_bound) ? 2.f * e_bound * 1.001f + 1e-30f : INFINITY;
             }
         }
 
         Sel S;
         S.init(ring + etid * 16, ring + kCandValBytes + etid * 4, ring + kCandBytes + etid * 4, zone_w);
-        STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_fold = 0; long long st_twait = 0, st_tfold = 0;
+        STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_fold = 0, st_miss = 0, st_nlat = 0; long long st_lat = 0; long long st_twait = 0, st_tfold = 0, st_tresc = 0, st_tfall = 0;
              const long long st_t0 = clock64();)
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
 
-        // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate scan
+        // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate append.  Straight-line
+        // code: the four predicated appends run whether or not any token of the warp has a candidate.  A warp-wide test
+        // that skips them would save issue slots in half of the chunks, but a warp's loop is a chain of latencies, and
+        // a vote plus a branch per chunk lengthens exactly that chain.
         auto process = [&](float (&v)[16], int col0) {
-            if (col0 + 16 > p.M) {                           // ragged end of the expert axis (warp-uniform)
-#pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (col0 + i >= p.M) v[i] = -INFINITY;
-            }
             float t[4];
 #pragma unroll
             for (int i = 0; i < 4; ++i) t[i] = fmaxf(max3(v[4 * i], v[4 * i + 1], v[4 * i + 2]), v[4 * i + 3]);
-            const float cmax = fmaxf(max3(t[0], t[1], t[2]), t[3]);
             if (LSE) {
+                const float cmax = fmaxf(max3(t[0], t[1], t[2]), t[3]);
                 const float c2 = cmax * kLog2e;
                 if (c2 > m2) { zsum *= ex2f(m2 - c2); m2 = c2; }
                 float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
@@ -573,59 +622,102 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 zsum += (a0 + a1) + (a2 + a3);
             }
             STAT(st_chunks++;)
-            if (__any_sync(kFullMask, cmax > S.thr)) {
-                STAT(st_hit++; const uint32_t mark = S.ptr;)
-                S.scan(v, t, col0);
-                STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
-                if (__any_sync(kFullMask, S.ptr >= S.warn)) {      // some token is about to run out of slots
-                    STAT(st_fold++; const long long tr0 = clock64();)
-                    S.fold();
-                    STAT(st_tfold += clock64() - tr0;)
-                }
+#ifdef MORE_EXP_NOSCAN
+            m2 = fmaxf(m2, t[0] + t[1] + t[2] + t[3]);
+            return;
+#endif
+            S.scan(v, t, col0);
+        };
+        // ---- after the two chunks of a buffer: fold if some token of the warp could overflow on the next buffer
+        auto fold_check = [&]() {
+            if (__any_sync(kFullMask, S.ptr >= S.warn)) {
+                STAT(st_fold++; const long long tr0 = clock64();)
+                S.fold();
+                STAT(st_tfold += clock64() - tr0;)
             }
         };
 
-        // ---- the sweep: buffer n of the group lives in ring slot n % NBUF
+        // ---- the sweep: buffer n of the group lives in ring slot n % NBUF.  A warp's loop is a chain of long
+        // latencies (barrier test, tensor-memory load), so it is software-pipelined: the second half of a buffer is in
+        // flight while the first is processed, the first half of the next buffer while the second is, and the buffer
+        // is handed back (this warp counted out of it) as soon as both halves are in registers.
+        // Refills take turns: the warp whose index in the group is n mod (live warps) refills buffer n's slot with
+        // buffer n + NBUF, one iteration later, when normally every warp has already counted itself out of it.  (Letting
+        // whichever warp is out last refill at once keeps the slowest warp the slowest; a separate issuing warp per
+        // group would exceed the thread count that leaves 96 registers per thread.)
         if (nb > 0 && ok) {
-            float va[16], vb[16];
-            STAT(const long long tw0 = clock64();)
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + g * 3), 0, abort_flag, p.status));
-            STAT(st_twait += clock64() - tw0;)
-            if (ok) {
-                tc_fence_after();
-                tmem_ld16(t_ring, va);
-            }
+            int slot = 0, pslot = 0, all_out = lw;                 // `released` reads all_out once every warp is out
+            int my_refill = q + 1;                                 // next iteration at which this warp refills a slot
             uint32_t ph = 0;
-            for (int n0 = 0; n0 < nb && ok; n0 += NBUF, ph ^= 1) {
+            const uint32_t rel0 = smem_u32(released + g * 3);
+            // One iteration = one buffer.  `masked` (a compile-time flag, so that the common iterations carry none of
+            // the masking code) is set for the buffers that reach beyond the range's end.  The two register buffers
+            // live inside one iteration only.
+            auto one_buffer = [&](auto masked, int n) {
+                const int col0 = e_lo + n * kBufCols;
+                float va[16], vb[16];
+                STAT(const long long tw1 = clock64(); if (!mbar_try_wait_now(bar(B_ACCF + g * 3 + slot), ph)) st_miss++;)
+                ok = mbar_wait(bar(B_ACCF + g * 3 + slot), ph, abort_flag, p.status);
+                STAT(st_twait += clock64() - tw1;)
+                if (!ok) return;
+                tc_fence_after();
+                tmem_ld16(t_ring + slot * kBufCols, va);
+                tmem_ld_wait16(va);
+                tmem_ld16(t_ring + slot * kBufCols + 16, vb);
+                if constexpr (decltype(masked)::value) {
 #pragma unroll
-                for (int s = 0; s < NBUF; ++s) {
-                    const int n = n0 + s;
-                    if (n < nb && ok) {
-                        const int col0 = e_lo + n * kBufCols;
-                        tmem_ld_wait16(va);
-                        tmem_ld16(t_ring + s * kBufCols + 16, vb);
-                        process(va, col0);
-                        tmem_ld_wait16(vb);
-                        tc_fence_before();
-                        warp_arrive(bar(B_ACCE + g * 3 + s), lane);          // the buffer is in registers: hand it back
-                        if (n + 1 < nb) {
-                            const int s1 = (s + 1) % NBUF;
-                            const uint32_t ph1 = (s + 1 == NBUF) ? (ph ^ 1) : ph;
-                            STAT(const long long tw1 = clock64();)
-                            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + g * 3 + s1), ph1, abort_flag, p.status));
-                            STAT(st_twait += clock64() - tw1;)
-                            if (ok) {
-                                tc_fence_after();
-                                tmem_ld16(t_ring + s1 * kBufCols, va);
-                            }
+                    for (int i = 0; i < 16; ++i)
+                        if (col0 + i >= e_hi) va[i] = -INFINITY;
+                }
+                process(va, col0);
+                STAT(const long long tl0 = clock64();)
+                tmem_ld_wait16(vb);
+                STAT(st_lat += clock64() - tl0; st_nlat++;)
+                // count this warp out of buffer n (release: its tensor-memory loads are complete)
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(rel0 + 4 * slot) : "memory");
+                // this warp's turn to refill the slot of buffer n - 1?  (all_out still counts buffer n - 1's use of it
+                // unless the slot index has just wrapped, in which case the count was raised one iteration early)
+                if (n == my_refill) {
+                    my_refill += lw;
+                    if (n - 1 + NBUF < nb) {
+                        const int want = (slot == 0) ? all_out - lw : all_out;
+                        const uint32_t ra = rel0 + 4 * pslot;
+                        int have, spins = 0;
+                        do {
+                            asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(have) : "r"(ra) : "memory");
+                        } while (have < want && ++spins < (1 << 26) && *abort_flag == 0);
+                        ok = have >= want;
+                        if (!ok) {
+                            if (*abort_flag == 0) { *abort_flag = 1; atomicExch(p.status, MORE_ERR_TIMEOUT); }
+                            return;
                         }
-                        process(vb, col0 + 16);
+                        tc_fence_after();
+                        ok = issue_buffer(g, b_lo0, n - 1 + NBUF, pslot);
+                        if (!ok) return;
                     }
                 }
-            }
+                if constexpr (decltype(masked)::value) {
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (col0 + 16 + i >= e_hi) vb[i] = -INFINITY;
+                }
+                process(vb, col0 + 16);
+                fold_check();
+                pslot = slot;
+                if (++slot == NBUF) { slot = 0; ph ^= 1; all_out += lw; }
+            };
+            const int ragged_from = min(nb, (e_hi - e_lo) / kBufCols);      // first buffer with columns to mask
+            int n = 0;
+            for (; n < ragged_from && ok; ++n) one_buffer(std::false_type{}, n);
+            for (; n < nb && ok; ++n) one_buffer(std::true_type{}, n);
+            ok = __all_sync(kFullMask, ok);
         }
         if (warp_live) S.fold();
         TopList<KCAP>& L = S.L;
+        STAT(const long long st_t1 = clock64();)
 
         if (FILTER && warp_live && ok) {
             // ---- rescoring: fp32 logits of the list and of the zone from the full z = hi + lo and the experts'
@@ -639,15 +731,17 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
             for (int e = 0; e < KCAP; ++e) acc[e] = 0.f;
             auto z_chunk = [&](int c, float (&z8)[8]) {             // ranks 8c .. 8c+7 of this token's z
-                uint32_t h4[4], l4[4];
+                uint32_t h4[4];
                 tmem_ld4(t_zop + c * 4, h4);
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(l4[0]), "=r"(l4[1]), "=r"(l4[2]), "=r"(l4[3])
-                             : "r"(zlo_addr + c * (kEpiThreads * 16)) : "memory");
+                const uint4 lv = zlo[c * kEpiThreads];
+                const uint32_t l4[4] = {lv.x, lv.y, lv.z, lv.w};
                 tmem_ld_wait4(h4);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    z8[2 * e] = bf_lo(h4[e]) + bf_lo(l4[e]);
-                    z8[2 * e + 1] = bf_hi(h4[e]) + bf_hi(l4[e]);
+                    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&h4[e]));
+                    const float2 lf = __half22float2(*reinterpret_cast<const __half2*>(&l4[e]));
+                    z8[2 * e] = (hf.x + lf.x) * zscale;
+                    z8[2 * e + 1] = (hf.y + lf.y) * zscale;
                 }
             };
             auto dot8 = [&](float a, const float (&z8)[8], const uint4& w) {
@@ -687,16 +781,34 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             }
             L = F;
         }
+        STAT(st_tresc = clock64() - st_t1;)
 #ifdef MORE_STATS
-        if (lane == 0 && p.stats && warp_live) {
+        if (p.stats && warp_live) {
+          const unsigned st_ov = __popc(__ballot_sync(kFullMask, FILTER && S.overflow && row_live));
+          const unsigned st_zn = __reduce_add_sync(kFullMask, (S.zptr - S.zbase) / kZoneStride);
+          if (lane == 0) {
             atomicAdd(p.stats + 0, (unsigned long long)st_chunks);
             atomicAdd(p.stats + 1, (unsigned long long)st_hit);
             atomicAdd(p.stats + 3, (unsigned long long)st_app);
             atomicAdd(p.stats + 4, (unsigned long long)st_fold);
             atomicAdd(p.stats + 8, (unsigned long long)st_twait);
-            atomicAdd(p.stats + 10, (unsigned long long)(clock64() - st_t0));
+            atomicAdd(p.stats + 9, (unsigned long long)st_miss);
+            atomicAdd(p.stats + 6, (unsigned long long)st_lat);
+            atomicAdd(p.stats + 5, (unsigned long long)st_nlat);
+            atomicAdd(p.stats + 4 + 0 * 1, 0ull);
+            atomicAdd(p.stats + 1 * 0 + 15 * 0 + 0, 0ull);
+            atomicAdd(p.stats + 15 - 15 + 0, 0ull);
+            atomicAdd(p.stats + 7 - 7 + 0, 0ull);
+            atomicAdd(p.stats + 10 - 10, 0ull);
+            atomicAdd(p.stats + 13 + (q >> 1), (unsigned long long)st_twait);
+            atomicAdd(p.stats + 15, (unsigned long long)(q >> 1));
+            atomicAdd(p.stats + 10, (unsigned long long)(st_t1 - st_t0));
+            atomicAdd(p.stats + 7, (unsigned long long)st_tresc);
+            atomicAdd(p.stats + 5, (unsigned long long)st_ov);
+            atomicAdd(p.stats + 2, (unsigned long long)st_zn);
             atomicAdd(p.stats + 11, 1ull);
             atomicAdd(p.stats + 12, (unsigned long long)st_tfold);
+          }
         }
 #endif
 
@@ -728,16 +840,18 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     // the token's z: the high part comes from tensor memory, which only whole warps can read
                     if (warp_live && __any_sync(kFullMask, slot >= 0)) {
                         for (int c = 0; c < RPAD / 8; ++c) {
-                            uint32_t h4[4], l4[4];
+                            uint32_t h4[4];
                             tmem_ld4(t_zop + c * 4, h4);
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(l4[0]), "=r"(l4[1]), "=r"(l4[2]), "=r"(l4[3])
-                                         : "r"(zlo_addr + c * (kEpiThreads * 16)) : "memory");
+                            const uint4 lv = zlo[c * kEpiThreads];
+                            const uint32_t l4[4] = {lv.x, lv.y, lv.z, lv.w};
                             tmem_ld_wait4(h4);
                             if (slot >= 0) {
 #pragma unroll
                                 for (int e = 0; e < 4; ++e) {
-                                    fz[slot * RPAD + c * 8 + 2 * e] = bf_lo(h4[e]) + bf_lo(l4[e]);
-                                    fz[slot * RPAD + c * 8 + 2 * e + 1] = bf_hi(h4[e]) + bf_hi(l4[e]);
+                                    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&h4[e]));
+                                    const float2 lf = __half22float2(*reinterpret_cast<const __half2*>(&l4[e]));
+                                    fz[slot * RPAD + c * 8 + 2 * e] = (hf.x + lf.x) * zscale;
+                                    fz[slot * RPAD + c * 8 + 2 * e + 1] = (hf.y + lf.y) * zscale;
                                 }
                             }
                         }
@@ -906,33 +1020,40 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 }
 
 // ------------------------------------------------------------------------------------ preparation (filter mode)
-// For the filter: R2T[j][i] = R2[i][j] (bf16, [M][RPAD], ranks >= r zero), the largest Euclidean column norm of R2
-// (slightly inflated, so that rounding cannot make it too small), and out_counts cleared.  One CTA per 64 experts;
+// For the filter: R2H = R2 converted to fp16 (same [r][M] layout, the B operand of the sweep), R2T[j][i] = R2[i][j]
+// (bf16, [M][RPAD], ranks >= r zero, for the rescoring), the largest Euclidean column norm of R2 and of R2 - R2H
+// (slightly inflated, so that rounding cannot make them too small), and out_counts cleared.  One CTA per 64 experts;
 // the CTA that finishes last reduces the per-CTA maxima (the arrival counter returns to zero for the next call).
 __global__ void __launch_bounds__(256)
-route_prepare_kernel(const __nv_bfloat16* __restrict__ R2, int r, int rpad, int M, __nv_bfloat16* __restrict__ r2t,
-                     float* __restrict__ partial, float* __restrict__ colnorm_max, unsigned* __restrict__ arrivals,
-                     int32_t* __restrict__ out_counts)
+route_prepare_kernel(const __nv_bfloat16* __restrict__ R2, int r, int rpad, int M, __half* __restrict__ r2h,
+                     __nv_bfloat16* __restrict__ r2t, float2* __restrict__ partial, float* __restrict__ colnorm,
+                     unsigned* __restrict__ arrivals, int32_t* __restrict__ out_counts)
 {
     __shared__ __nv_bfloat16 tile[64][64 + 8];      // [rank][expert], padded rows
-    __shared__ float red[64];
+    __shared__ float red[64], rederr[64];
     __shared__ int last;
     const int j0 = blockIdx.x * 64;
     const int tj = threadIdx.x & 63, ti = threadIdx.x >> 6;
     for (int i = ti; i < rpad; i += 4) {
         __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-        if (i < r && j0 + tj < M) v = R2[(int64_t)i * M + j0 + tj];
+        if (i < r && j0 + tj < M) {
+            v = R2[(int64_t)i * M + j0 + tj];
+            r2h[(int64_t)i * M + j0 + tj] = __float2half_rn(__bfloat162float(v));
+        }
         tile[i][tj] = v;
     }
     if (threadIdx.x < 64 && j0 + threadIdx.x < M) out_counts[j0 + threadIdx.x] = 0;
     __syncthreads();
     if (threadIdx.x < 64) {
-        float s = 0.f;
+        float s = 0.f, se = 0.f;
         for (int i = 0; i < rpad; ++i) {
             const float x = __bfloat162float(tile[i][threadIdx.x]);
+            const float e = x - __half2float(__float2half_rn(x));       // +-inf if x overflows fp16
             s = fmaf(x, x, s);
+            se = fmaf(e, e, se);
         }
         red[threadIdx.x] = s;
+        rederr[threadIdx.x] = se;
     }
     // transposed rows: 16 bytes (8 ranks) per item
     const int chunks = rpad / 8;
@@ -949,23 +1070,29 @@ route_prepare_kernel(const __nv_bfloat16* __restrict__ R2, int r, int rpad, int 
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        float m = 0.f;
-        for (int i = 0; i < 64; ++i) m = fmaxf(m, red[i]);
-        partial[blockIdx.x] = m;
+        float m = 0.f, me = 0.f;
+        for (int i = 0; i < 64; ++i) { m = fmaxf(m, red[i]); me = fmaxf(me, rederr[i]); }
+        partial[blockIdx.x] = make_float2(m, me);
         __threadfence();
         last = (atomicAdd(arrivals, 1u) == gridDim.x - 1);
     }
     __syncthreads();
     if (last) {
         __threadfence();
-        float m = 0.f;
-        for (int i = threadIdx.x; i < (int)gridDim.x; i += 256) m = fmaxf(m, __ldcg(partial + i));
-        __shared__ float red2[256];
+        float m = 0.f, me = 0.f;
+        for (int i = threadIdx.x; i < (int)gridDim.x; i += 256) {
+            const float2 v = __ldcg(partial + i);
+            m = fmaxf(m, v.x);
+            me = fmaxf(me, v.y);
+        }
+        __shared__ float red2[256], red3[256];
         red2[threadIdx.x] = m;
+        red3[threadIdx.x] = me;
         __syncthreads();
         if (threadIdx.x == 0) {
-            for (int i = 1; i < 256; ++i) m = fmaxf(m, red2[i]);
-            *colnorm_max = sqrtf(m) * 1.0001f;
+            for (int i = 1; i < 256; ++i) { m = fmaxf(m, red2[i]); me = fmaxf(me, red3[i]); }
+            colnorm[0] = sqrtf(m) * 1.0001f;
+            colnorm[1] = sqrtf(me) * 1.0001f;      // NaN-free: me >= 0, possibly +inf
             *arrivals = 0;
         }
     }
@@ -1015,7 +1142,7 @@ int rpad_of(int r) { return r <= 16 ? 16 : (r <= 32 ? 32 : 64); }
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct ScratchLayout {
-    size_t counters, part_val, part_id, part_mz, r2t, partial, total;
+    size_t counters, part_val, part_id, part_mz, r2t, r2h, partial, zlo, total;
 };
 
 ScratchLayout scratch_layout(const RouteArgs& a, const Plan& p)
@@ -1033,7 +1160,9 @@ ScratchLayout scratch_layout(const RouteArgs& a, const Plan& p)
     }
     if (p.filter) {
         L.r2t = off; off += align_up((size_t)a.M * rpad_of(a.r) * 2, 256);
-        L.partial = off; off += align_up((size_t)((a.M + 63) / 64) * 4, 256);
+        L.r2h = off; off += align_up((size_t)a.M * a.r * 2, 256);
+        L.partial = off; off += align_up((size_t)((a.M + 63) / 64) * 8, 256);
+        L.zlo = off; off += align_up((size_t)p.ctas * (rpad_of(a.r) / 8) * kEpiThreads * 16, 256);
     }
     L.total = off;
     return L;
@@ -1054,13 +1183,14 @@ bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st
                        int* r2_off)
 {
     const int st2 = es * rpad * 128;
-    const int fixed = kCandBytes + (filter ? kZoneBytes + kEpiThreads * rpad * 2 : 0);
+    const int fixed = kCandBytes + (filter ? kZoneBytes : 0);
     int n2 = (kRRing - fixed) / st2;
-    if (n2 > 8) n2 = 8;
+    n2 = n2 >= 8 ? 8 : (n2 >= 4 ? 4 : n2);                  // a power of two (the kernel masks step numbers with it)
     const int st1 = tg * kXGroupBytes + kR1Bytes;
     // phase 1 wants at least two stages below the R2 stages
-    while (n2 > 2 && kRRing - n2 * st2 < 2 * st1) --n2;
+    while (n2 > 2 && kRRing - n2 * st2 < 2 * st1) n2 /= 2;
     if (n2 < 2) return false;
+    if (n2 == 3) n2 = 2;
     const int off = (kRRing - n2 * st2) & ~1023;
     int n1 = off / st1;
     if (n1 > 4) n1 = 4;
@@ -1075,10 +1205,13 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     RouteParams rp{};
     if (!lowrank_smem_plan(rpad, p.tg, p.es, p.filter, &rp.nst1, &rp.st1_bytes, &rp.nst2, &rp.st2_bytes, &rp.r2_off))
         return MORE_ERR_SHAPE;
+    const ScratchLayout L = scratch_layout(a, p);
+    char* base = static_cast<char*>(scratch);
     CUtensorMap mx, m1, m2;
     int rc = get_tensor_map(a.X, a.T, a.h, 128, 64, &mx);
     if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
-    if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.r, a.M, rpad, 64, &m2);
+    // the filter sweeps the fp16 copy of R2 in scratch (same shape; a 16-bit type either way as far as TMA cares)
+    if (rc == MORE_OK) rc = get_tensor_map(p.filter ? static_cast<const void*>(base + L.r2h) : a.R2, a.r, a.M, rpad, 64, &m2);
     if (rc != MORE_OK) return rc;
 
     rp.T = a.T; rp.h = a.h; rp.r = a.r; rp.M = a.M; rp.k = a.k; rp.gate_mode = a.gate_mode;
@@ -1090,8 +1223,6 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     rp.status = ctx.status;
     rp.stats = ctx.stats;
     rp.R2 = a.R2;
-    const ScratchLayout L = scratch_layout(a, p);
-    char* base = static_cast<char*>(scratch);
     if (p.msplit > 1) {
         rp.counters = reinterpret_cast<unsigned*>(base + L.counters);
         rp.part_val = reinterpret_cast<float*>(base + L.part_val);
@@ -1114,11 +1245,13 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     if (p.filter) {
         __nv_bfloat16* r2t = reinterpret_cast<__nv_bfloat16*>(base + L.r2t);
         rp.r2t = r2t;
-        rp.colnorm_max = ctx.colnorm_max;
+        rp.colnorm = ctx.colnorm;
+        rp.zlo = reinterpret_cast<uint4*>(base + L.zlo);
         // the preparation kernel also clears out_counts
-        route_prepare_kernel<<<(a.M + 63) / 64, 256, 0, a.stream>>>(a.R2, a.r, rpad, a.M, r2t,
-                                                                   reinterpret_cast<float*>(base + L.partial),
-                                                                   ctx.colnorm_max, ctx.prep_arrivals, a.out_counts);
+        route_prepare_kernel<<<(a.M + 63) / 64, 256, 0, a.stream>>>(a.R2, a.r, rpad, a.M,
+                                                                   reinterpret_cast<__half*>(base + L.r2h), r2t,
+                                                                   reinterpret_cast<float2*>(base + L.partial),
+                                                                   ctx.colnorm, ctx.prep_arrivals, a.out_counts);
         count_launch(1);
         if (cudaGetLastError() != cudaSuccess) return MORE_ERR_CUDA;
     } else if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) {

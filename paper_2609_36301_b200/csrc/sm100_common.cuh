@@ -55,6 +55,20 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok;
 }
 
+// Non-blocking test of a phase.
+__device__ __forceinline__ uint32_t mbar_try_wait_now(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+
 // Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of budget).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
 {
@@ -299,7 +313,50 @@ __host__ __device__ constexpr uint32_t umma_idesc(int n)
     return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
            ((uint32_t)(128 >> 4) << 24);
 }
+// The same with A = B = fp16 (format code 0).
+__host__ __device__ constexpr uint32_t umma_idesc_f16(int n)
+{
+    return (1u << 4) | (0u << 7) | (0u << 10) | (0u << 15) | (1u << 16) | ((uint32_t)(n >> 3) << 17) |
+           ((uint32_t)(128 >> 4) << 24);
+}
 
+// All MMAs of one accumulator buffer in a single instruction sequence: D[128 x N] = sum over NM K-steps of
+// A (tensor memory, 8 columns per K = 16 step) x B (shared memory, MN-major, 16 K-rows = 2048 bytes per step; the B
+// offset wraps after KS steps, which is how a [hi | lo] operand pair reuses the same B rows).  The warp executes it
+// converged; one elected lane issues.  b_lo / b_hi are the two words of the B descriptor.
+#define MORE_MMA_STEP(AOFF, BOFF, PRED)                                                              \
+    "add.u32 a, %1, " #AOFF ";\n\tadd.u32 bl, %2, " #BOFF ";\n\tmov.b64 bd, {bl, %3};\n\t"        \
+    "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], [a], bd, %4, " #PRED ";\n\t"
+#define MORE_MMA_OPEN                                                                                \
+    "{\n\t.reg .pred pe, pt, pf;\n\t.reg .b64 bd;\n\t.reg .b32 a, bl;\n\t"                        \
+    "setp.eq.u32 pt, 0, 0;\n\tsetp.ne.u32 pf, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+template <int NM, int KS>
+__device__ __forceinline__ void tc_mma_buffer_ts(uint32_t d, uint32_t a0, uint32_t b_lo, uint32_t b_hi, uint32_t idesc)
+{
+    static_assert((NM == 1 && KS == 1) || (NM == 2 && (KS == 1 || KS == 2)) || (NM == 4 && (KS == 2 || KS == 4)) ||
+                  (NM == 8 && KS == 4), "unsupported MMA sequence");
+    if constexpr (NM == 1)
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) "}" ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else if constexpr (NM == 2 && KS == 2)
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) MORE_MMA_STEP(8, 128, pt) "}"
+                     ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else if constexpr (NM == 2 && KS == 1)
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) MORE_MMA_STEP(8, 0, pt) "}"
+                     ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else if constexpr (NM == 4 && KS == 4)
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) MORE_MMA_STEP(8, 128, pt) MORE_MMA_STEP(16, 256, pt)
+                     MORE_MMA_STEP(24, 384, pt) "}" ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else if constexpr (NM == 4 && KS == 2)
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) MORE_MMA_STEP(8, 128, pt) MORE_MMA_STEP(16, 0, pt)
+                     MORE_MMA_STEP(24, 128, pt) "}" ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else
+        asm volatile(MORE_MMA_OPEN MORE_MMA_STEP(0, 0, pf) MORE_MMA_STEP(8, 128, pt) MORE_MMA_STEP(16, 256, pt)
+                     MORE_MMA_STEP(24, 384, pt) MORE_MMA_STEP(32, 0, pt) MORE_MMA_STEP(40, 128, pt)
+                     MORE_MMA_STEP(48, 256, pt) MORE_MMA_STEP(56, 384, pt) "}"
+                     ::"r"(d), "r"(a0), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+}
+#undef MORE_MMA_STEP
+#undef MORE_MMA_OPEN
 
 }  // namespace
 
