@@ -52,6 +52,7 @@ struct Plan {
     int tg = 1;   // low-rank router: 128-token groups per CTA ...
     int es = 1;   // ... and expert ranges swept side by side inside a CTA (tg * es <= 4)
     bool filter = false;   // low-rank router: approximate sweep + exact rescoring of the survivors
+    bool paired = false;   // low-rank router: the kernel with 256-token CTAs, two per SM, instead of one CTA per SM
 };
 
 bool tcgen05_shape_ok(int T, int h, int r, int M, int k);
@@ -65,12 +66,16 @@ bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st
 size_t generic_scratch_bytes(const RouteArgs& a);
 size_t lowrank_scratch_bytes(const RouteArgs& a, const Plan& p);
 size_t full_scratch_bytes(const RouteArgs& a, const Plan& p);
+size_t paired_scratch_bytes(const RouteArgs& a, const Plan& p);
 
 // Launchers: enqueue on a.stream, return MORE_OK / MORE_ERR_*.  `scratch` is at least *_scratch_bytes().
 int launch_generic(const RouteArgs& a, DeviceCtx& ctx, void* scratch);
 // Both tensor-core launchers clear out_counts on the stream themselves, after every host-side step that can fail.
 int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
 int launch_full(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
+int launch_paired(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch);
+// Filter mode's preparation: fp16 copy and transposed copy of R2, column-norm maxima, out_counts cleared.
+int launch_route_prepare(const RouteArgs& a, int rpad, void* r2h, void* r2t, void* partial, DeviceCtx& ctx);
 
 int launch_generic_psum(const __nv_bfloat16* X, const __nv_bfloat16* R1, const __nv_bfloat16* R2, int T, int h, int r,
                         int M, const float* lse, float* psum, void* scratch, cudaStream_t stream);

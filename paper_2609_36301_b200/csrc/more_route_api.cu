@@ -86,8 +86,10 @@ int route_device_locked(const RouteArgs& a, int path, int msplit)
     const bool want_lse = a.gate_mode == MORE_GATE_FULL_SOFTMAX || a.out_lse != nullptr;
     rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, want_lse, a.full, path, msplit, ctx->sm_count, &plan);
     if (rc != MORE_OK) return rc;
-    const size_t need = plan.path != MORE_PATH_TCGEN05 ? generic_scratch_bytes(a)
-                                                       : (a.full ? full_scratch_bytes(a, plan) : lowrank_scratch_bytes(a, plan));
+    const size_t need = plan.path != MORE_PATH_TCGEN05
+                            ? generic_scratch_bytes(a)
+                            : (a.full ? full_scratch_bytes(a, plan)
+                                      : (plan.paired ? paired_scratch_bytes(a, plan) : lowrank_scratch_bytes(a, plan)));
     rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, need);
     if (rc != MORE_OK) return rc;
     if (a.T == 0 || plan.path != MORE_PATH_TCGEN05) {
@@ -96,7 +98,8 @@ int route_device_locked(const RouteArgs& a, int path, int msplit)
         if (a.T == 0) return MORE_OK;
         return launch_generic(a, *ctx, ctx->scratch);
     }
-    return a.full ? launch_full(a, *ctx, plan, ctx->scratch) : launch_lowrank(a, *ctx, plan, ctx->scratch);
+    if (a.full) return launch_full(a, *ctx, plan, ctx->scratch);
+    return plan.paired ? launch_paired(a, *ctx, plan, ctx->scratch) : launch_lowrank(a, *ctx, plan, ctx->scratch);
 }
 
 int route_device(const RouteArgs& a, int path, int msplit)
@@ -154,7 +157,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
 {
     const int blocks64 = (M + 63) / 64;
     const int rpad = r <= 16 ? 16 : (r <= 32 ? 32 : 64);
-    const bool filter_ok = !want_lse && k <= 16 && M >= 4096;
+    const bool filter_ok = false;      // (the filter mode is built and tested but is not faster on any measured shape)
     const double c_lat = want_lse ? 260.0 : 190.0, c_iss = want_lse ? 120.0 : 62.0;
     double best = 1e300;
     Plan bp = *p;
@@ -167,7 +170,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
             if (!lowrank_smem_plan(rpad, tg, es, filter_ok, &n1, &b1, &n2, &b2, &off)) continue;
             int s_lo = 1, s_hi = 1;
             if (msplit > 0) {
-                s_lo = s_hi = msplit;
+                s_lo = s_hi = msplit < blocks64 / es ? msplit : (blocks64 / es > 0 ? blocks64 / es : 1);   // at most one CTA per 64-expert block
             } else {
                 s_hi = sm_count / blocks;                      // never more CTAs than one wave
                 if (s_hi > blocks64 / (es * 8)) s_hi = blocks64 / (es * 8);    // a range keeps at least 512 experts
@@ -221,16 +224,31 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
     if (full) {
         plan_full(T, h, M, msplit, sm_count, &p);
     } else {
+        // Two kernels serve the low-rank router (measured on B200, both gate modes, T from 8 k to 64 k tokens): the
+        // grouped kernel (one CTA per SM, up to four token groups / expert ranges side by side) wins while an SM has
+        // fewer than ~160 tokens, and up to ~320 tokens per SM when no softmax sweep is wanted and the expert count is
+        // moderate; the paired kernel (256-token CTAs, two per SM, 64-expert steps) wins on everything larger.
         p.block_tokens = 0;
-        plan_lowrank(T, h, r, M, k, want_lse, msplit, sm_count, &p);
+        const long long per_sm = ((long long)T + sm_count - 1) / sm_count;
+        bool grouped = per_sm < 160 || (!want_lse && per_sm < 320 && M <= 32768);
+#ifdef MORE_DEV
+        if (const char* kk = getenv("MORE_KERNEL")) grouped = kk[0] == 'g';
+#endif
+        if (grouped) {
+            plan_lowrank(T, h, r, M, k, want_lse, msplit, sm_count, &p);
+        } else {
+            plan_full(T, h, M, msplit, sm_count, &p);
+            p.paired = true;
+        }
         if (p.block_tokens == 0) return MORE_ERR_SHAPE;
 #ifdef MORE_DEV
-        // development builds only: MORE_PLAN="block_tokens,es,msplit,filter" overrides the planner
+        // development builds only: MORE_PLAN="block_tokens,es,msplit,filter[,paired]" overrides the planner
         if (const char* e = getenv("MORE_PLAN")) {
-            int bt = 0, es = 0, s = 0, f = 0;
-            if (sscanf(e, "%d,%d,%d,%d", &bt, &es, &s, &f) == 4) {
+            int bt = 0, es = 0, s = 0, f = 0, pr = 0;
+            if (sscanf(e, "%d,%d,%d,%d,%d", &bt, &es, &s, &f, &pr) >= 4) {
                 p.block_tokens = bt; p.tg = (bt + 127) / 128; p.es = es; p.msplit = s;
                 p.filter = f != 0 && !want_lse && k <= 16;
+                p.paired = pr != 0;
                 p.ctas = ((T + bt - 1) / bt) * s;
             }
         }

@@ -31,7 +31,9 @@
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device
 // status word, raises the CTA's abort flag and all roles fall through to the common exit (TMEM is freed there).
 #include "sm100_common.cuh"
+#include "more_select.cuh"
 
+#include <cuda_fp16.h>
 #include <limits.h>
 
 // -DMORE_STATS builds count epilogue events and clocks into KernelParams::stats (diagnostics only).
@@ -45,95 +47,10 @@ namespace more {
 
 namespace {
 
-// Running top-k of one token.  Between refreshes the sorted list is left alone.  A chunk of 16 logits is looked at
-// as four groups of four; every group whose maximum beats the cached threshold `tau` (the list's last entry as of
-// the last refresh, hence never above the true threshold) is appended whole, in ascending column order, to this
-// thread's column of a shared-memory candidate buffer: one predicated 16-byte store of the four values (they sit in
-// four consecutive registers as loaded from tensor memory, so nothing is moved), one predicated 4-byte store of the
-// group's first column into a parallel array, and no branch.  refresh() then inserts the buffered elements that beat
-// the up-to-date threshold, so the inserts of several chunks of all 32 tokens of a warp are executed together.  A
-// chunk appends at most 4 entries and the warp refreshes as soon as some token has fewer than 4 free slots left, so
-// the buffer cannot overflow.
-constexpr int kCandValStride = kEpilogueThreads * 16;     // bytes between successive value slots of one thread
-constexpr int kCandColStride = kEpilogueThreads * 4;      // ... and between its column slots
 #ifndef MORE_CAND_CAP
 #define MORE_CAND_CAP 8
 #endif
-constexpr unsigned kFullMask = 0xffffffffu;
-
-template <int KCAP, int CAP>
-struct Selector {
-    static constexpr int kWarnSlots = CAP - 4;            // a chunk must always find 4 free slots
-    static_assert(kWarnSlots >= 1, "candidate buffer too small");
-    TopList<KCAP> L;
-    float tau;
-    uint32_t ptr;     // shared-memory address of this thread's next free value slot
-    uint32_t cptr;    // ... and of the matching column slot
-    uint32_t base, cbase;
-    uint32_t warn;    // at or beyond this fill level the warp refreshes after the chunk
-
-    __device__ __forceinline__ void init(uint32_t first_val_slot, uint32_t first_col_slot)
-    {
-        L.init();
-        tau = -INFINITY;
-        base = ptr = first_val_slot;
-        cbase = cptr = first_col_slot;
-        warn = first_val_slot + kWarnSlots * kCandValStride;
-    }
-    // Called by all 32 lanes of a warp together.  Every round inserts at most one element per token: the maximum
-    // of the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
-    // (rising) threshold any more moves on to its next entries.  The rounds end when no token has anything left, so
-    // their number is the largest count of real insertions of any token of the warp, and the (select-only) insert
-    // code is executed once per round.
-    __device__ __forceinline__ void refresh()
-    {
-        uint32_t a = base, c = cbase;
-        float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
-        int col = 0;
-        for (;;) {
-            float m = fmaxf(max3(x0, x1, x2), x3);
-            while (!(m > L.tau()) && a < ptr) {
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(a) : "memory");
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(col) : "r"(c) : "memory");
-                a += kCandValStride;
-                c += kCandColStride;
-                m = fmaxf(max3(x0, x1, x2), x3);
-            }
-            const bool pass = m > L.tau();
-            if (!__any_sync(kFullMask, pass)) break;
-            // the maximum's lowest column on a tie, so that equal logits enter the list in ascending column order
-            const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : ((x2 == m) ? 2 : 3));
-            if (pass) L.insert(m, col + j);
-            x0 = (j == 0) ? -INFINITY : x0;
-            x1 = (j == 1) ? -INFINITY : x1;
-            x2 = (j == 2) ? -INFINITY : x2;
-            x3 = (j == 3) ? -INFINITY : x3;
-        }
-        ptr = base;
-        cptr = cbase;
-        tau = L.tau();
-    }
-    // if (t > tau) append {v0, v1, v2, v3} and col
-    __device__ __forceinline__ void append4(float t, float v0, float v1, float v2, float v3, int col)
-    {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.gt.f32 p, %2, %8;\n\t"
-            "@p st.shared.v4.b32 [%0], {%3, %4, %5, %6};\n\t"
-            "@p st.shared.b32 [%1], %7;\n\t"
-            "@p add.u32 %0, %0, %9;\n\t"
-            "@p add.u32 %1, %1, %10;\n\t}"
-            : "+r"(ptr), "+r"(cptr)
-            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "f"(v3), "r"(col), "f"(tau), "n"(kCandValStride), "n"(kCandColStride)
-            : "memory");
-    }
-    // v: 16 logits of columns col0.., t: maxima of the groups (v[4i] .. v[4i+3]).
-    __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[4], int col0)
-    {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) append4(t[i], v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3], col0 + 4 * i);
-    }
-};
+constexpr int kFallbackSlots = 8;      // tokens re-routed per round of the filter's fallback (one per epilogue warp)
 
 struct KernelParams {
     int T, h, r, M, k, gate_mode, msplit;
@@ -152,6 +69,13 @@ struct KernelParams {
     float* part_val;
     int* part_id;
     float2* part_mz;
+    // filter mode: transposed copy of R2 ([M][RPAD] bf16, ranks >= r zero); colnorm[0] = largest column norm of R2,
+    // colnorm[1] = largest column norm of the error of its fp16 copy; R2 itself for the fallback sweep; the low halves
+    // of z, [CTA][rank / 8][256 threads] x 16 B
+    const __nv_bfloat16* r2t;
+    const float* colnorm;
+    const __nv_bfloat16* R2;
+    uint4* zlo;
 };
 
 // Final outputs of one token from its sorted list and (m2, z): m2 is the running max in log2 units.
@@ -189,7 +113,13 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
 // contraction running over K = h): there is no phase 1, every 64-expert step instead accumulates over all h/64 k-tiles
 // of X (256 x 64, re-read per step) and W (64 x 64) with the phase-1 pipeline and stage layout, and the epilogue is
 // the same.  map_r2 is then W's map (64 x 64 boxes), map_r1 is unused, RPAD is 64.
-template <int RPAD, int KCAP, bool LSE, bool FULL = false>
+//
+// FILTER = true (low-rank router, top-k-softmax gate, no log-sum-exp): the second contraction runs on one fp16 rounding
+// of z (scaled per token by a power of two) against an fp16 copy of R2, i.e. half the MMAs; the selection keeps every
+// expert within W = 2E of the running k-th approximate logit, E bounding what the rounding can change, and the
+// survivors are rescored in fp32 from the full z and the transposed copy of R2; a token whose zone store overflows is
+// routed again by a plain sweep.  The result is the exact top-k of the fp32 logits either way.
+template <int RPAD, int KCAP, bool LSE, bool FULL = false, bool FILTER = false>
 __global__ void __launch_bounds__(kThreads, 2)
 route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_r1,
                      const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
@@ -199,9 +129,12 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
     // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
     constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
-    using Sel = Selector<KCAP, kCandCap>;
-    constexpr int kCandValBytes = kCandCap * kCandValStride;
-    constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);
+    using Sel = Selector<KCAP, FILTER, kEpilogueThreads, kCandCap, 4>;
+    constexpr int kCandValStride = Sel::kCandValStride;
+    constexpr int kCandValBytes = Sel::kCandValBytes;
+    constexpr int kZoneOff = Sel::kCandBytes;                     // filter: the zone store follows the candidates
+    constexpr int kCandBytes = Sel::kCandBytes + (FILTER ? Sel::kZoneBytes : 0);
+    constexpr int kMmas2 = FILTER ? kKSteps : 2 * kKSteps;      // exact modes: hi then lo into one accumulator
     // R2 blocks in flight: what the ring has room for next to the candidate buffers, at most 8 (unused by FULL)
     constexpr int kStagesFit = (kRingBytes - kCandBytes) / kR2StageBytes;
     constexpr int kStagesP2 = FULL ? 1 : (kStagesFit < 8 ? kStagesFit : 8);
@@ -227,6 +160,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
+    int* flagged = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 12);      // filter: tokens that need the fallback sweep
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
@@ -252,6 +186,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads / 2); }
         *abort_flag = 0;
         *last_flag = 0;
+        *flagged = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -312,7 +247,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // The whole warp runs this code converged; one elected lane issues each tcgen05 instruction.
         bool ok = true;
         constexpr uint32_t idesc1 = umma_idesc(64);
-        constexpr uint32_t idesc2 = umma_idesc(kHalf);
+        constexpr uint32_t idesc2 = FILTER ? umma_idesc_f16(kHalf) : umma_idesc(kHalf);
         if constexpr (FULL) {
             // standard router: per 64-expert step, K runs over all of h through the two k-tile stages
             const uint64_t xd = umma_desc_sw128(ring, 16, 1024), wd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
@@ -386,7 +321,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int j = 0; j < 2 * kKSteps; ++j)       // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
+                for (int j = 0; j < kMmas2; ++j)            // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
                     tc_mma_bf16_ts_elect(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64 + j * 8,
                                          b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
                 tc_commit_elect(bar(B_ACCF + a));
@@ -409,9 +344,31 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         STAT(const long long st_k0 = clock64();)
         bool ok = FULL ? true : mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
         STAT(const long long st_k1 = clock64();)
+        const int etid0 = threadIdx.x - 64;                  // 0..255 among the epilogue threads
+        // filter: low half of this thread's z, 16 B per 8 ranks, in global scratch (read back once, for rescoring)
+        uint4* zlo = FILTER ? p.zlo + (size_t)blockIdx.x * (RPAD / 8) * kEpilogueThreads + etid0 : nullptr;
+        float zone_w = 0.f, zscale = 1.f;                    // filter: zone width; z = (hi + lo) * zscale
         if (ok && !FULL) {
-            // ---- narrow z to bf16 [hi | lo] and store it to tensor memory as the A operand of phase 2
+            // ---- narrow z and store it to tensor memory as the A operand of phase 2: bf16 [hi | lo], or (filter) z
+            // scaled by a power of two and rounded to fp16
             tc_fence_after();
+            float lo2 = 0.f, z2 = 0.f, down = 1.f;
+            if (FILTER) {
+                // power of two that brings the token's largest |z| into [2^13, 2^14)
+                float zmax = 0.f;
+#pragma unroll
+                for (int c = 0; c < RPAD / 16; ++c) {
+                    float z[16];
+                    tmem_ld16(t_lane + c * 16, z);
+                    tmem_ld_wait16(z);
+#pragma unroll
+                    for (int e = 0; e < 16; ++e) zmax = fmaxf(zmax, fabsf(z[e]));
+                }
+                int ex = (int)((__float_as_uint(zmax) >> 23) & 0xffu) - 127;      // floor(log2 zmax) for normal zmax
+                ex = (zmax > 0.f && zmax < INFINITY) ? max(-100, min(100, ex - 13)) : 0;
+                zscale = __uint_as_float((uint32_t)(127 + ex) << 23);
+                down = __uint_as_float((uint32_t)(127 - ex) << 23);
+            }
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
@@ -420,22 +377,52 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 uint32_t hi[8], lo[8];
 #pragma unroll
                 for (int e = 0; e < 8; ++e) {
-                    const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
-                    const __nv_bfloat16 l0 = __float2bfloat16_rn(z[2 * e] - __bfloat162float(h0));
-                    const __nv_bfloat16 l1 = __float2bfloat16_rn(z[2 * e + 1] - __bfloat162float(h1));
-                    hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
-                    lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                    if (FILTER) {
+                        const float z0 = z[2 * e] * down, z1 = z[2 * e + 1] * down;
+                        const __half2 h = __floats2half2_rn(z0, z1);
+                        const float2 hf = __half22float2(h);
+                        const float d0 = z0 - hf.x, d1 = z1 - hf.y;
+                        const __half2 l = __floats2half2_rn(d0, d1);
+                        hi[e] = *reinterpret_cast<const uint32_t*>(&h);
+                        lo[e] = *reinterpret_cast<const uint32_t*>(&l);
+                        // the part of z the approximate logits do not see, and the size of z itself
+                        lo2 = fmaf(d0, d0, lo2);
+                        lo2 = fmaf(d1, d1, lo2);
+                        z2 = fmaf(z0, z0, z2);
+                        z2 = fmaf(z1, z1, z2);
+                    } else {
+                        const __nv_bfloat16 h0 = __float2bfloat16_rn(z[2 * e]), h1 = __float2bfloat16_rn(z[2 * e + 1]);
+                        const __nv_bfloat16 l0 = __float2bfloat16_rn(z[2 * e] - __bfloat162float(h0));
+                        const __nv_bfloat16 l1 = __float2bfloat16_rn(z[2 * e + 1] - __bfloat162float(h1));
+                        hi[e] = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+                        lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+                    }
                 }
                 tmem_st8(t_zop + c * 8, hi);
-                tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                if (FILTER) {
+                    zlo[(2 * c) * kEpilogueThreads] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                    zlo[(2 * c + 1) * kEpilogueThreads] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                } else {
+                    tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                }
             }
             tmem_st_wait();
             tc_fence_before();
             mbar_arrive(bar(B_ZOP));
+            if (FILTER) {
+                // |approximate - fp32 logit| (both in the scaled units of this token) <= |z - hi|_2 |R2_j|_2 for the
+                // part of z the sweep does not see, + |z|_2 |R2_j - fp16(R2_j)|_2 for what the fp16 copy of R2 lost,
+                // + the accumulation rounding of the two evaluations, bounded by 2^-18 |z|_2 |R2_j|_2 (a generous
+                // multiple of fp32 epsilon).
+                const float cn = __ldg(p.colnorm), cerr = __ldg(p.colnorm + 1);
+                const float e_bound = sqrtf(lo2) * cn * 1.001f + sqrtf(z2) * (cn * 3.8147e-6f + cerr * 1.001f);
+                // (e_bound is zero only for z = 0, where every logit is exactly zero either way)
+                zone_w = (e_bound == e_bound) ? 2.f * e_bound * 1.001f : INFINITY;
+            }
         }
 
         Sel S;
-        S.init(cand + row_in_blk * 16, cand + kCandValBytes + row_in_blk * 4);
+        S.init(cand + row_in_blk * 16, cand + kCandValBytes + row_in_blk * 4, cand + kZoneOff + row_in_blk * 4, zone_w);
         STAT(unsigned st_chunks = 0, st_hit = 0, st_app = 0, st_rcall = 0, st_riter = 0; long long st_twait = 0, st_tproc = 0, st_tref = 0;
              const long long st_t0 = clock64();)
         float m2 = -INFINITY, zsum = 0.f;                    // running max (log2 units) and sum of 2^(y - m2)
@@ -482,14 +469,14 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 m2 = fmaxf(m2, cmax);
                 return;
 #endif
-                if (__any_sync(kFullMask, cmax > S.tau)) {
+                if (__any_sync(kFullMask, cmax > S.thr)) {
                     STAT(st_hit++; const uint32_t mark = S.ptr;)
                     S.scan(v, t, col0);
                     STAT(st_app += __reduce_add_sync(kFullMask, (S.ptr - mark) / kCandValStride);)
                     if (__any_sync(kFullMask, S.ptr >= S.warn)) {
                         // some token is about to run out of slots: fold now
                         STAT(st_rcall++; const long long tr0 = clock64();)
-                        S.refresh();
+                        S.fold();
                         STAT(st_tref += clock64() - tr0;)
                     }
                 }
@@ -522,8 +509,71 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             process(vb, e0 + 48);
             STAT(st_tproc += clock64() - tw1;)
         }
-        S.refresh();
+        S.fold();
         TopList<KCAP>& L = S.L;
+
+        if (FILTER && warp_live && group_live && ok) {
+            // ---- rescoring: fp32 logits of the list and of the zone from the full z = (hi + lo) * zscale and the
+            // experts' columns (rows of the transposed copy of R2); the exact values decide the final order
+            S.prune();
+            const int zcount = (int)((S.zptr - S.zbase) / Sel::kZoneStride);
+            int zmax = zcount;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) zmax = max(zmax, __shfl_xor_sync(kFullMask, zmax, o));
+            float acc[KCAP];
+#pragma unroll
+            for (int e = 0; e < KCAP; ++e) acc[e] = 0.f;
+            auto z_chunk = [&](int c, float (&z8)[8]) {             // ranks 8c .. 8c+7 of this token's z
+                uint32_t h4[4];
+                tmem_ld4(t_zop + c * 4, h4);
+                const uint4 lv = zlo[c * kEpilogueThreads];
+                const uint32_t l4[4] = {lv.x, lv.y, lv.z, lv.w};
+                tmem_ld_wait4(h4);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&h4[e]));
+                    const float2 lf = __half22float2(*reinterpret_cast<const __half2*>(&l4[e]));
+                    z8[2 * e] = (hf.x + lf.x) * zscale;
+                    z8[2 * e + 1] = (hf.y + lf.y) * zscale;
+                }
+            };
+            auto dot8 = [&](float a, const float (&z8)[8], const uint4& w) {
+                a = fmaf(z8[0], bf_lo(w.x), a); a = fmaf(z8[1], bf_hi(w.x), a);
+                a = fmaf(z8[2], bf_lo(w.y), a); a = fmaf(z8[3], bf_hi(w.y), a);
+                a = fmaf(z8[4], bf_lo(w.z), a); a = fmaf(z8[5], bf_hi(w.z), a);
+                a = fmaf(z8[6], bf_lo(w.w), a); a = fmaf(z8[7], bf_hi(w.w), a);
+                return a;
+            };
+            const uint4* r2t = reinterpret_cast<const uint4*>(p.r2t);
+            for (int c = 0; c < RPAD / 8; ++c) {
+                float z8[8];
+                z_chunk(c, z8);
+#pragma unroll
+                for (int e = 0; e < KCAP; ++e) {
+                    if ((unsigned)L.id[e] < (unsigned)p.M) {
+                        const uint4 w = __ldg(r2t + (size_t)L.id[e] * (RPAD / 8) + c);
+                        acc[e] = dot8(acc[e], z8, w);
+                    }
+                }
+            }
+            TopList<KCAP> F;
+            F.init();
+#pragma unroll
+            for (int e = 0; e < KCAP; ++e)
+                if ((unsigned)L.id[e] < (unsigned)p.M) F.insert_ordered(acc[e], L.id[e]);
+            for (int zi = 0; zi < zmax; ++zi) {
+                const bool have = zi < zcount;
+                const int id = have ? lds_s32(S.zbase + Sel::kZoneIdOff + zi * Sel::kZoneStride) : -1;
+                float a = 0.f;
+                for (int c = 0; c < RPAD / 8; ++c) {
+                    float z8[8];
+                    z_chunk(c, z8);
+                    if ((unsigned)id < (unsigned)p.M) a = dot8(a, z8, __ldg(r2t + (size_t)id * (RPAD / 8) + c));
+                }
+                if ((unsigned)id < (unsigned)p.M) F.insert_ordered(a, id);
+            }
+            L = F;
+        }
 #ifdef MORE_STATS
         if (lane == 0 && p.stats) {
             atomicAdd(p.stats + 0, (unsigned long long)st_chunks);
@@ -548,8 +598,63 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // memory and flushes only the non-zero bins with one global atomic each; otherwise straight to global memory
         // (with that many experts the bins hardly collide).  With few experts thousands of pairs hit each bin, and
         // same-address global atomics would serialise.
-        int* hist = (p.M * 4 <= kRingBytes) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
         const int etid = threadIdx.x - 64;                   // 0..255 among the epilogue threads
+        if constexpr (FILTER) {
+            // ---- fallback: tokens whose zone overflowed are routed again, exactly, over this CTA's experts; the result
+            // replaces the token's list.  Rounds of kFallbackSlots tokens, one warp per token.
+            auto epi_sync = [&]() { asm volatile("bar.sync 1, 256;" ::: "memory"); };
+            if (S.overflow && row_live) atomicAdd(flagged, 1);
+            epi_sync();
+            const int nflag = (*abort_flag == 0) ? *flagged : 0;
+            if (nflag > 0) {
+                float* fz = reinterpret_cast<float*>(ring_ptr);                          // [slot][RPAD] z
+                float* fv = fz + kFallbackSlots * RPAD;                                   // [slot][KCAP]
+                int* fi = reinterpret_cast<int*>(fv + kFallbackSlots * KCAP);
+                int* ticket = fi + kFallbackSlots * KCAP;
+                if (etid == 0) *ticket = 0;
+                epi_sync();
+                bool mine = S.overflow && row_live;
+                for (int done = 0; done < nflag; done += kFallbackSlots) {
+                    int slot = -1;
+                    if (mine) {
+                        const int t = atomicAdd(ticket, 1);
+                        if (t < done + kFallbackSlots) slot = t - done; else atomicSub(ticket, 1);
+                    }
+                    // the token's z: the high part comes from tensor memory, which only whole warps can read
+                    if (warp_live && group_live && __any_sync(kFullMask, slot >= 0)) {
+                        for (int c = 0; c < RPAD / 8; ++c) {
+                            uint32_t h4[4];
+                            tmem_ld4(t_zop + c * 4, h4);
+                            const uint4 lv = zlo[c * kEpilogueThreads];
+                            const uint32_t l4[4] = {lv.x, lv.y, lv.z, lv.w};
+                            tmem_ld_wait4(h4);
+                            if (slot >= 0) {
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const float2 hf = __half22float2(*reinterpret_cast<const __half2*>(&h4[e]));
+                                    const float2 lf = __half22float2(*reinterpret_cast<const __half2*>(&l4[e]));
+                                    fz[slot * RPAD + c * 8 + 2 * e] = (hf.x + lf.x) * zscale;
+                                    fz[slot * RPAD + c * 8 + 2 * e + 1] = (hf.y + lf.y) * zscale;
+                                }
+                            }
+                        }
+                    }
+                    epi_sync();
+                    const int nslots = min(kFallbackSlots, nflag - done);
+                    if (warp - 2 < nslots)
+                        exact_topk_warp<KCAP>(fz + (warp - 2) * RPAD, p.R2, p.r, p.M, e_lo, e_hi, fv + (warp - 2) * KCAP,
+                                              fi + (warp - 2) * KCAP, lane);
+                    epi_sync();
+                    if (slot >= 0) {
+#pragma unroll
+                        for (int e = 0; e < KCAP; ++e) { L.v[e] = fv[slot * KCAP + e]; L.id[e] = fi[slot * KCAP + e]; }
+                        mine = false;
+                    }
+                    epi_sync();
+                }
+            }
+        }
+        int* hist = (p.M <= kRingBytes / 4) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
         auto hist_clear = [&]() {
             if (hist) {
                 for (int e = etid; e < p.M; e += kEpilogueThreads) hist[e] = 0;
@@ -716,12 +821,12 @@ int get_tensor_map(const void* ptr, int rows, int cols, int box_rows, int box_co
 
 namespace {
 
-template <int RPAD, int KCAP, bool LSE, bool FULL>
+template <int RPAD, int KCAP, bool LSE, bool FULL, bool FILTER>
 int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp, int ctas,
-               cudaStream_t st)
+               cudaStream_t st, bool clear_counts)
 {
     static unsigned long long configured = 0;   // one bit per device, per instantiation; guarded by the API mutex
-    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE, FULL>;
+    auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE, FULL, FILTER>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (!(configured >> (dev & 63) & 1ull)) {
@@ -730,77 +835,131 @@ int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& 
         configured |= 1ull << (dev & 63);
     }
     // every host-side step that can fail is behind us: only now is the first output touched
-    if (cudaMemsetAsync(kp.out_counts, 0, (size_t)kp.M * sizeof(int32_t), st) != cudaSuccess) return MORE_ERR_CUDA;
+    if (clear_counts &&
+        cudaMemsetAsync(kp.out_counts, 0, (size_t)kp.M * sizeof(int32_t), st) != cudaSuccess)
+        return MORE_ERR_CUDA;
     kern<<<ctas, kThreads, kSmemBytes, st>>>(mx, m1, m2, kp);
     count_launch(1);
     return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
 }
 
+// mode: 0 exact, 1 exact with the softmax sweep, 2 filter
 template <int RPAD, int KCAP, bool FULL>
-int launch_lse(bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp,
-               int ctas, cudaStream_t st)
+int launch_mode(int mode, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2, const KernelParams& kp,
+                int ctas, cudaStream_t st, bool clear_counts)
 {
-    return lse ? launch_one<RPAD, KCAP, true, FULL>(mx, m1, m2, kp, ctas, st)
-               : launch_one<RPAD, KCAP, false, FULL>(mx, m1, m2, kp, ctas, st);
+    if (mode == 1) return launch_one<RPAD, KCAP, true, FULL, false>(mx, m1, m2, kp, ctas, st, clear_counts);
+    if (mode == 0) return launch_one<RPAD, KCAP, false, FULL, false>(mx, m1, m2, kp, ctas, st, clear_counts);
+    if constexpr (!FULL && KCAP <= 16) return launch_one<RPAD, KCAP, false, false, true>(mx, m1, m2, kp, ctas, st, clear_counts);
+    else return MORE_ERR_SHAPE;
 }
 
 template <int RPAD, bool FULL>
-int launch_kcap(int k, bool lse, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2,
-                const KernelParams& kp, int ctas, cudaStream_t st)
+int launch_kcap(int k, int mode, const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& m2,
+                const KernelParams& kp, int ctas, cudaStream_t st, bool clear_counts)
 {
-    if (k <= 8) return launch_lse<RPAD, 8, FULL>(lse, mx, m1, m2, kp, ctas, st);
-    if (k <= 16) return launch_lse<RPAD, 16, FULL>(lse, mx, m1, m2, kp, ctas, st);
-    return launch_lse<RPAD, 32, FULL>(lse, mx, m1, m2, kp, ctas, st);
+    if (k <= 8) return launch_mode<RPAD, 8, FULL>(mode, mx, m1, m2, kp, ctas, st, clear_counts);
+    if (k <= 16) return launch_mode<RPAD, 16, FULL>(mode, mx, m1, m2, kp, ctas, st, clear_counts);
+    return launch_mode<RPAD, 32, FULL>(mode, mx, m1, m2, kp, ctas, st, clear_counts);
 }
 
 int kcap_of(int k) { return k <= 8 ? 8 : (k <= 16 ? 16 : 32); }
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-}  // namespace
+struct PairedScratch {
+    size_t counters, part_val, part_id, part_mz, r2t, r2h, partial, zlo, total;
+};
 
-size_t full_scratch_bytes(const RouteArgs& a, const Plan& p)
+PairedScratch paired_layout(const RouteArgs& a, const Plan& p)
 {
-    if (p.msplit <= 1) return 0;
-    const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
-    const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
-    const size_t kc = (size_t)kcap_of(a.k);
-    return align_up(blocks * 4, 256) + align_up(slots * kc * 4, 256) * 2 + align_up(slots * 8, 256);
+    PairedScratch L{};
+    size_t off = 0;
+    if (p.msplit > 1) {
+        const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
+        const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
+        const size_t kc = (size_t)kcap_of(a.k);
+        L.counters = off; off += align_up(blocks * 4, 256);
+        L.part_val = off; off += align_up(slots * kc * 4, 256);
+        L.part_id = off; off += align_up(slots * kc * 4, 256);
+        L.part_mz = off; off += align_up(slots * 8, 256);
+    }
+    if (p.filter) {
+        const size_t rpad = a.r <= 16 ? 16 : (a.r <= 32 ? 32 : 64);
+        L.r2t = off; off += align_up((size_t)a.M * rpad * 2, 256);
+        L.r2h = off; off += align_up((size_t)a.M * a.r * 2, 256);
+        L.partial = off; off += align_up((size_t)((a.M + 63) / 64) * 8, 256);
+        L.zlo = off; off += align_up((size_t)p.ctas * (rpad / 8) * kEpilogueThreads * 16, 256);
+    }
+    L.total = off;
+    return L;
 }
 
-int launch_full(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
+}  // namespace
+
+size_t full_scratch_bytes(const RouteArgs& a, const Plan& p) { return paired_layout(a, p).total; }
+size_t paired_scratch_bytes(const RouteArgs& a, const Plan& p) { return paired_layout(a, p).total; }
+
+// The kernel of this file for either router: the fused standard router (a.full) or the low-rank router with 256-token
+// CTAs, two per SM ("paired": two 128-token groups per CTA).
+int launch_paired(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
 {
-    CUtensorMap mx, m2;
-    int rc = get_tensor_map(a.X, a.T, a.h, kBlockTokens, 64, &mx);
-    // W [h][M]: its k-tiles are 64 x 64 boxes
-    if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.h, a.M, 64, 64, &m2);
+    const PairedScratch L = paired_layout(a, p);
+    char* base = static_cast<char*>(scratch);
+    const int rpad = a.full ? 64 : (a.r <= 16 ? 16 : (a.r <= 32 ? 32 : 64));
+    const int x_rows = (!a.full && p.block_tokens <= 128) ? 128 : kBlockTokens;
+    CUtensorMap mx, m1, m2;
+    int rc = get_tensor_map(a.X, a.T, a.h, x_rows, 64, &mx);
+    if (a.full) {
+        // W [h][M]: its k-tiles are 64 x 64 boxes
+        if (rc == MORE_OK) rc = get_tensor_map(a.R2, a.h, a.M, 64, 64, &m2);
+        m1 = m2;
+    } else {
+        if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
+        // the filter sweeps the fp16 copy of R2 in scratch (same shape; a 16-bit type either way as far as TMA cares)
+        if (rc == MORE_OK)
+            rc = get_tensor_map(p.filter ? static_cast<const void*>(base + L.r2h) : a.R2, a.r, a.M, rpad, 64, &m2);
+    }
     if (rc != MORE_OK) return rc;
 
-    KernelParams kp;
+    KernelParams kp{};
     kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
     kp.block_tokens = p.block_tokens;
-    kp.x_rows = kBlockTokens;
+    kp.x_rows = x_rows;
     kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
     kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
     kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
     kp.status = ctx.status;
     kp.stats = ctx.stats;
-    kp.counters = nullptr; kp.part_val = nullptr; kp.part_id = nullptr; kp.part_mz = nullptr;
+    kp.R2 = a.R2;
     if (p.msplit > 1) {
+        kp.counters = reinterpret_cast<unsigned*>(base + L.counters);
+        kp.part_val = reinterpret_cast<float*>(base + L.part_val);
+        kp.part_id = reinterpret_cast<int*>(base + L.part_id);
+        kp.part_mz = reinterpret_cast<float2*>(base + L.part_mz);
         const size_t blocks = (size_t)(a.T + p.block_tokens - 1) / p.block_tokens;
-        const size_t slots = blocks * kBlockTokens * (size_t)p.msplit;
-        const size_t kc = (size_t)kcap_of(a.k);
-        char* base = static_cast<char*>(scratch);
-        kp.counters = reinterpret_cast<unsigned*>(base);
-        base += align_up(blocks * 4, 256);
-        kp.part_val = reinterpret_cast<float*>(base);
-        base += align_up(slots * kc * 4, 256);
-        kp.part_id = reinterpret_cast<int*>(base);
-        base += align_up(slots * kc * 4, 256);
-        kp.part_mz = reinterpret_cast<float2*>(base);
         if (cudaMemsetAsync(kp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
     }
     const bool lse = (a.gate_mode == MORE_GATE_FULL_SOFTMAX) || (a.out_lse != nullptr);
-    return launch_kcap<64, true>(a.k, lse, mx, m2, m2, kp, p.ctas, a.stream);
+    int mode = lse ? 1 : 0;
+    if (p.filter) {
+        if (lse || a.k > 16 || a.full) return MORE_ERR_SHAPE;
+        mode = 2;
+        kp.r2t = reinterpret_cast<const __nv_bfloat16*>(base + L.r2t);
+        kp.colnorm = ctx.colnorm;
+        kp.zlo = reinterpret_cast<uint4*>(base + L.zlo);
+        // the preparation kernel also clears out_counts
+        rc = launch_route_prepare(a, rpad, base + L.r2h, base + L.r2t, base + L.partial, ctx);
+        if (rc != MORE_OK) return rc;
+    }
+    const bool clear = !p.filter;
+    if (a.full) return launch_kcap<64, true>(a.k, mode, mx, m1, m2, kp, p.ctas, a.stream, clear);
+    switch (rpad) {
+        case 16: return launch_kcap<16, false>(a.k, mode, mx, m1, m2, kp, p.ctas, a.stream, clear);
+        case 32: return launch_kcap<32, false>(a.k, mode, mx, m1, m2, kp, p.ctas, a.stream, clear);
+        default: return launch_kcap<64, false>(a.k, mode, mx, m1, m2, kp, p.ctas, a.stream, clear);
+    }
 }
+
+int launch_full(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch) { return launch_paired(a, ctx, p, scratch); }
 
 }  // namespace more

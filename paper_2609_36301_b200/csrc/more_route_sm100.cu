@@ -49,6 +49,7 @@
 // Every mbarrier wait is bounded: when the budget runs out the thread records MORE_ERR_TIMEOUT in the device status
 // word, raises the CTA's abort flag and all roles fall through to the common exit (tensor memory is freed there).
 #include "sm100_common.cuh"
+#include "more_select.cuh"
 
 #include <cuda_fp16.h>
 
@@ -76,18 +77,16 @@ constexpr int kBufCols = 32;                       // one accumulator buffer of 
 #define MORE_CAND_CAP 12
 #endif
 constexpr int kCandCap = MORE_CAND_CAP;            // candidate slots per token
-constexpr int kCandValStride = kEpiThreads * 16;   // bytes between successive value slots of one thread
-constexpr int kCandColStride = kEpiThreads * 4;    // ... and between its column slots
-constexpr int kCandValBytes = kCandCap * kCandValStride;
-constexpr int kCandBytes = kCandCap * (kCandValStride + kCandColStride);      // 80 KB
-constexpr int kZoneCap = 8;                        // zone slots per token (filter mode)
-constexpr int kZoneStride = kEpiThreads * 4;
-constexpr int kZoneIdOff = kZoneCap * kZoneStride;
-constexpr int kZoneBytes = 2 * kZoneIdOff;         // 32 KB
+using SelLayout = Selector<8, true, kEpiThreads, kCandCap, 8>;      // (byte layout only: independent of KCAP, FILTER)
+constexpr int kCandValStride = SelLayout::kCandValStride;
+constexpr int kCandValBytes = SelLayout::kCandValBytes;
+constexpr int kCandBytes = SelLayout::kCandBytes;
+constexpr int kZoneStride = SelLayout::kZoneStride;
+constexpr int kZoneIdOff = SelLayout::kZoneIdOff;
+constexpr int kZoneBytes = SelLayout::kZoneBytes;
 constexpr int kXGroupBytes = 128 * 128;            // X tile of one token group: 128 tokens x 64 bf16
 constexpr int kR1Bytes = 64 * 128;
 constexpr int kFallbackSlots = 16;                 // tokens re-routed per round of the fallback (one per epilogue warp)
-constexpr unsigned kFullMask = 0xffffffffu;
 constexpr float kLog2e = 1.4426950408889634f;
 
 enum { kModeExact = 0, kModeExactLse = 1, kModeFilter = 2 };
@@ -117,148 +116,6 @@ struct RouteParams {
     const float* colnorm;
     const __nv_bfloat16* R2;     // for the fallback sweep
     uint4* zlo;                  // filter: the low halves of z, [CTA][rank / 8][512 threads] x 16 B
-};
-
-// ---------------------------------------------------------------------------------------- shared-memory access
-__device__ __forceinline__ float lds_f32(uint32_t a)
-{
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ int lds_s32(uint32_t a)
-{
-    int v;
-    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(a) : "memory");
-    return v;
-}
-__device__ __forceinline__ void sts_f32(uint32_t a, float v) { asm volatile("st.shared.f32 [%0], %1;" ::"r"(a), "f"(v) : "memory"); }
-__device__ __forceinline__ void sts_s32(uint32_t a, int v) { asm volatile("st.shared.b32 [%0], %1;" ::"r"(a), "r"(v) : "memory"); }
-__device__ __forceinline__ float bf_lo(uint32_t u) { return __uint_as_float(u << 16); }
-__device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
-
-// Running top-k of one token.  Between folds the sorted list is left alone.  A chunk of 16 logits is looked at as four
-// groups of four; every group whose maximum beats the cached threshold `thr` (never above the true one) is appended
-// whole, in ascending column order, to this thread's column of a shared-memory candidate buffer: one predicated
-// 16-byte store of the four values (they sit in four consecutive registers as loaded from tensor memory), one
-// predicated 4-byte store of the group's first column, no branch.  fold() then inserts the buffered elements that beat
-// the up-to-date threshold, so the inserts of several chunks of all 32 tokens of a warp are executed together.  A chunk
-// appends at most 4 entries and the warp folds as soon as some token has fewer than 4 free slots left, so the buffer
-// cannot overflow.
-//
-// FILTER: the logits are approximate to within E; thr sits W = 2E below the list's last value, elements that land in
-// that zone (directly, or pushed out of the list) are kept in a second small per-token store, pruned when it fills
-// up; a token whose zone still overflows is flagged for the fallback.
-template <int KCAP, bool FILTER>
-struct Selector {
-    TopList<KCAP> L;
-    float thr;
-    float W;
-    uint32_t ptr, cptr, base, cbase, warn;
-    uint32_t zptr, zbase;
-    bool overflow;
-
-    __device__ __forceinline__ void init(uint32_t first_val_slot, uint32_t first_col_slot, uint32_t first_zone_slot, float w)
-    {
-        L.init();
-        thr = -INFINITY;
-        W = w;
-        base = ptr = first_val_slot;
-        cbase = cptr = first_col_slot;
-        warn = first_val_slot + (kCandCap - 8) * kCandValStride;      // a 32-column buffer appends at most 8 entries
-        zbase = zptr = first_zone_slot;
-        overflow = false;
-    }
-    __device__ __forceinline__ float limit() const { return FILTER ? L.tau() - W : L.tau(); }
-
-    // Drop the zone entries that have fallen more than W below the list; flag the token if the zone is still full.
-    __device__ __forceinline__ void prune()
-    {
-        const float lim = limit();
-        uint32_t rd = zbase, wr = zbase;
-        while (__any_sync(kFullMask, rd < zptr)) {
-            const bool act = rd < zptr;
-            float v = -INFINITY;
-            int id = 0;
-            if (act) { v = lds_f32(rd); id = lds_s32(rd + kZoneIdOff); }
-            if (act && v > lim) {
-                sts_f32(wr, v);
-                sts_s32(wr + kZoneIdOff, id);
-                wr += kZoneStride;
-            }
-            rd += kZoneStride;
-        }
-        zptr = wr;
-        if (zptr >= zbase + kZoneCap * kZoneStride) { overflow = true; zptr = zbase; }
-    }
-
-    // Called by all 32 lanes of a warp together.  Every round handles at most one element per token: the maximum of
-    // the token's current entry, which is then struck out of the entry; a token whose entry holds nothing above its
-    // (rising) limit any more moves on to its next entries.  The rounds end when no token has anything left.
-    __device__ __forceinline__ void fold()
-    {
-#ifdef MORE_EXP_NOFOLD
-        ptr = base; cptr = cbase; thr = 3.2f; return;      // timing experiment: what the scan alone costs
-#endif
-        uint32_t a = base, c = cbase;
-        float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
-        int col = 0;
-        for (;;) {
-            float m = fmaxf(max3(x0, x1, x2), x3);
-            while (!(m > limit()) && a < ptr) {
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(a) : "memory");
-                col = lds_s32(c);
-                a += kCandValStride;
-                c += kCandColStride;
-                m = fmaxf(max3(x0, x1, x2), x3);
-            }
-            const bool pass = m > limit();
-            if (!__any_sync(kFullMask, pass)) break;
-            // the maximum's lowest column on a tie, so that equal logits enter the list in ascending column order
-            const int j = (x0 == m) ? 0 : ((x1 == m) ? 1 : ((x2 == m) ? 2 : 3));
-            if constexpr (FILTER) {
-                const bool ins = pass && (m > L.tau());
-                const float ev = ins ? L.v[KCAP - 1] : m;          // what may belong into the zone: the entry pushed
-                const int ei = ins ? L.id[KCAP - 1] : col + j;     // out of the list, or the element itself
-                if (ins) L.insert(m, col + j);
-                if (pass && ev > limit()) {
-                    sts_f32(zptr, ev);
-                    sts_s32(zptr + kZoneIdOff, ei);
-                    zptr += kZoneStride;
-                }
-                if (__any_sync(kFullMask, zptr >= zbase + kZoneCap * kZoneStride)) prune();
-            } else {
-                if (pass) L.insert(m, col + j);
-            }
-            x0 = (j == 0) ? -INFINITY : x0;
-            x1 = (j == 1) ? -INFINITY : x1;
-            x2 = (j == 2) ? -INFINITY : x2;
-            x3 = (j == 3) ? -INFINITY : x3;
-        }
-        ptr = base;
-        cptr = cbase;
-        thr = limit();
-    }
-    // if (t > thr) append {v0, v1, v2, v3} and col
-    __device__ __forceinline__ void append4(float t, float v0, float v1, float v2, float v3, int col)
-    {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "setp.gt.f32 p, %2, %8;\n\t"
-            "@p st.shared.v4.b32 [%0], {%3, %4, %5, %6};\n\t"
-            "@p st.shared.b32 [%1], %7;\n\t"
-            "@p add.u32 %0, %0, %9;\n\t"
-            "@p add.u32 %1, %1, %10;\n\t}"
-            : "+r"(ptr), "+r"(cptr)
-            : "f"(t), "f"(v0), "f"(v1), "f"(v2), "f"(v3), "r"(col), "f"(thr), "n"(kCandValStride), "n"(kCandColStride)
-            : "memory");
-    }
-    // v: 16 logits of columns col0.., t: maxima of the groups (v[4i] .. v[4i+3]).
-    __device__ __forceinline__ void scan(const float (&v)[16], const float (&t)[4], int col0)
-    {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) append4(t[i], v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3], col0 + 4 * i);
-    }
 };
 
 // Final outputs of one token from its sorted list and (m2, z): m2 is the running max in log2 units.
@@ -291,43 +148,6 @@ __device__ __forceinline__ void write_token(const RouteParams& p, int64_t row, c
     if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
 }
 
-// Exact top-KCAP of one token over experts [e_lo, e_hi) by a plain CUDA-core sweep, run by one warp: lane j takes the
-// experts e_lo + j, e_lo + j + 32, ..., computes each logit as the fp32 chain l = fma(z[i], R2[i][e], l) over i
-// ascending (the same chain the rescoring of the filter uses), keeps a lane-local sorted list, and the 32 lists are
-// merged by KCAP rounds of a warp-wide argmax under the full order (value descending, id ascending).  zs: the token's
-// z in shared memory (r floats); the result goes to out_v / out_id (shared memory, KCAP entries).
-template <int KCAP>
-__device__ __noinline__ void exact_topk_warp(const float* zs, const __nv_bfloat16* __restrict__ R2, int r, int M,
-                                             int e_lo, int e_hi, float* out_v, int* out_id, int lane)
-{
-    TopList<KCAP> L;
-    L.init();
-    for (int e = e_lo + lane; e < e_hi; e += 32) {
-        float l = 0.f;
-        for (int i = 0; i < r; ++i) l = fmaf(zs[i], __bfloat162float(R2[(int64_t)i * M + e]), l);
-        if (l > L.tau()) L.insert(l, e);
-    }
-    for (int q = 0; q < KCAP; ++q) {
-        float bv = L.v[0];
-        int bi = L.id[0];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-            const float ov = __shfl_xor_sync(kFullMask, bv, o);
-            const int oi = __shfl_xor_sync(kFullMask, bi, o);
-            const bool take = ov > bv || (ov == bv && oi < bi);
-            bv = take ? ov : bv;
-            bi = take ? oi : bi;
-        }
-        if (lane == 0) { out_v[q] = bv; out_id[q] = bi; }
-        if (L.id[0] == bi && L.v[0] == bv && bi != INT_MAX) {      // the winning lane pops its head
-#pragma unroll
-            for (int s = 0; s + 1 < KCAP; ++s) { L.v[s] = L.v[s + 1]; L.id[s] = L.id[s + 1]; }
-            L.v[KCAP - 1] = -INFINITY;
-            L.id[KCAP - 1] = INT_MAX;
-        }
-    }
-}
-
 // ------------------------------------------------------------------------------------------------- the kernel
 template <int RPAD, int KCAP, int MODE>
 __global__ void __launch_bounds__(kRThreads, 1)
@@ -342,7 +162,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kRingCol0 = (kZopCols <= 32) ? 32 : 64;            // first column of the accumulator ring
     constexpr int NBUF = (kGroupCols - kRingCol0) / kBufCols;        // 3 or 2
     constexpr int kR2BlockBytes = RPAD * 128;                        // RPAD rows x 64 experts
-    using Sel = Selector<KCAP, FILTER>;
+    using Sel = Selector<KCAP, FILTER, kEpiThreads, kCandCap, 8>;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -589,7 +409,8 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 // multiple of fp32 epsilon).
                 const float cn = __ldg(p.colnorm), cerr = __ldg(p.colnorm + 1);
                 const float e_bound = sqrtf(lo2) * cn * 1.001f + sqrtf(z2) * (cn * 3.8147e-6f + cerr * 1.001f);
-                zone_w = (e_bound == e_bound) ? 2.f * e_bound * 1.001f + 1e-30f : INFINITY;
+                // (e_bound is zero only for z = 0, where every logit is exactly zero either way)
+                zone_w = (e_bound == e_bound) ? 2.f * e_bound * 1.001f : INFINITY;
             }
         }
 
@@ -1199,6 +1020,16 @@ bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st
     return true;
 }
 
+int launch_route_prepare(const RouteArgs& a, int rpad, void* r2h, void* r2t, void* partial, DeviceCtx& ctx)
+{
+    route_prepare_kernel<<<(a.M + 63) / 64, 256, 0, a.stream>>>(a.R2, a.r, rpad, a.M, static_cast<__half*>(r2h),
+                                                               static_cast<__nv_bfloat16*>(r2t),
+                                                               static_cast<float2*>(partial), ctx.colnorm,
+                                                               ctx.prep_arrivals, a.out_counts);
+    count_launch(1);
+    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
+
 int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scratch)
 {
     const int rpad = rpad_of(a.r);
@@ -1243,17 +1074,12 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
         if (cudaMemsetAsync(rp.counters, 0, blocks * 4, a.stream) != cudaSuccess) return MORE_ERR_CUDA;
     }
     if (p.filter) {
-        __nv_bfloat16* r2t = reinterpret_cast<__nv_bfloat16*>(base + L.r2t);
-        rp.r2t = r2t;
+        rp.r2t = reinterpret_cast<const __nv_bfloat16*>(base + L.r2t);
         rp.colnorm = ctx.colnorm;
         rp.zlo = reinterpret_cast<uint4*>(base + L.zlo);
         // the preparation kernel also clears out_counts
-        route_prepare_kernel<<<(a.M + 63) / 64, 256, 0, a.stream>>>(a.R2, a.r, rpad, a.M,
-                                                                   reinterpret_cast<__half*>(base + L.r2h), r2t,
-                                                                   reinterpret_cast<float2*>(base + L.partial),
-                                                                   ctx.colnorm, ctx.prep_arrivals, a.out_counts);
-        count_launch(1);
-        if (cudaGetLastError() != cudaSuccess) return MORE_ERR_CUDA;
+        const int prc = launch_route_prepare(a, rpad, base + L.r2h, base + L.r2t, base + L.partial, ctx);
+        if (prc != MORE_OK) return prc;
     } else if (cudaMemsetAsync(a.out_counts, 0, (size_t)a.M * sizeof(int32_t), a.stream) != cudaSuccess) {
         return MORE_ERR_CUDA;
     }

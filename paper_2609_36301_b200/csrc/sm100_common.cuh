@@ -249,49 +249,6 @@ __device__ __forceinline__ void warp_arrive(uint32_t bar, int lane)
     if (lane == 0) mbar_arrive(bar);
 }
 
-// ---------------------------------------------------------------------------------------------- running top-k
-// Sorted (value, id) list of one token, held in registers.
-template <int KCAP>
-struct TopList {
-    float v[KCAP];
-    int id[KCAP];
-    __device__ __forceinline__ void init()
-    {
-#pragma unroll
-        for (int s = 0; s < KCAP; ++s) { v[s] = -INFINITY; id[s] = INT_MAX; }
-    }
-    __device__ __forceinline__ float tau() const { return v[KCAP - 1]; }
-    // Insert (x, j) with x > tau().  Equal values keep the earlier (smaller-id) entry ahead.
-    __device__ __forceinline__ void insert(float x, int j)
-    {
-#pragma unroll
-        for (int s = KCAP - 1; s > 0; --s) {
-            const bool above_prev = x > v[s - 1];
-            const bool above_this = x > v[s];
-            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
-            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
-        }
-        const bool top = x > v[0];
-        v[0] = top ? x : v[0];
-        id[0] = top ? j : id[0];
-    }
-    // Insert with the full order (value descending, id ascending): for merging lists whose ids interleave.
-    __device__ __forceinline__ void insert_ordered(float x, int j)
-    {
-        auto ahead = [&](int s) { return x > v[s] || (x == v[s] && j < id[s]); };
-#pragma unroll
-        for (int s = KCAP - 1; s > 0; --s) {
-            const bool above_prev = ahead(s - 1);
-            const bool above_this = ahead(s);
-            v[s] = above_prev ? v[s - 1] : (above_this ? x : v[s]);
-            id[s] = above_prev ? id[s - 1] : (above_this ? j : id[s]);
-        }
-        const bool top = ahead(0);
-        v[0] = top ? x : v[0];
-        id[0] = top ? j : id[0];
-    }
-};
-
 // ------------------------------------------------------------------------------------------- UMMA descriptors
 // Shared-memory matrix descriptor, 128-byte swizzle, descriptor version 1 (sm_100).
 //   K-major operand  (rows = M/N index, 128-byte rows of 64 bf16 along K): SBO = 1024 B between 8-row groups.

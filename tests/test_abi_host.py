@@ -61,10 +61,36 @@ def test_plan_picks_paths_and_splits():
     assert P(64, 64, 8, 260, 4).path == mr.PATH_GENERIC          # M % 8 != 0
     with pytest.raises(mr.MoreRouteError):
         P(100, 20, 5, 33, 3, path=mr.PATH_TCGEN05)
-    p = P(8192, 4096, 64, 131072, 16)
-    assert p.msplit > 1 and p.ctas % p.msplit == 0              # few token blocks, many experts: split the experts
-    assert 32 <= p.ctas // p.msplit <= 64 and p.ctas <= 296     # 128..256 tokens per CTA, one wave of 2 CTAs per SM
-    assert P(65536, 2048, 64, 16384, 8).ctas in range(256, 297)
-    assert P(32768, 512, 32, 1024, 8).msplit * 128 <= 1024      # never more CTAs per block than expert tiles
+    with pytest.raises(mr.MoreRouteError):
+        P(300, 256, 32, 4096, 8, msplit=65)                      # more than 64 CTAs per token block
+    PX = mr.more_route_plan_ex
+    # few token blocks, many experts: the experts are split, inside a CTA and over CTAs, and one wave is not exceeded
+    p = PX(8192, 4096, 64, 131072, 16, gate_mode=1)
+    assert p.ctas % p.msplit == 0 and p.ctas <= 148
+    assert p.msplit * p.expert_ranges >= 4 and p.token_groups * p.expert_ranges <= 4
+    # many tokens: the kernel with 256-token CTAs, two per SM, in one wave
+    p = PX(65536, 2048, 64, 16384, 8)
+    assert p.ctas in range(256, 297) and p.msplit == 1
+    # a decode-sized batch is spread over the SMs along the expert axis
+    p = PX(64, 2048, 64, 16384, 8)
+    assert p.ctas > 16 and p.ctas <= 148 and p.msplit > 1
+    # never more CTAs per token block than 64-expert blocks
+    assert PX(300, 256, 32, 256, 8, msplit=5).msplit * PX(300, 256, 32, 256, 8, msplit=5).expert_ranges <= 4
     assert P(300, 256, 32, 4096, 8, msplit=5).msplit == 5
-    assert P(300, 256, 32, 256, 8, msplit=5).msplit == 2        # clamped to the number of 128-expert tiles
+    # asking for the log-sum-exp changes the kernel variant but is always accepted
+    assert PX(32768, 512, 32, 16384, 8, want_lse=True).path == mr.PATH_TCGEN05
+
+
+def test_shared_memory_plan_of_the_grouped_kernel_fits():
+    """Every (rank, token groups, expert ranges) the planner may pick leaves room for at least two R2 stages and one
+    phase-1 stage in the 208 KB ring (checked through the plans of shapes that exercise them)."""
+    PX = mr.more_route_plan_ex
+    for T in (1, 33, 128, 200, 300, 512, 5000, 20000):
+        for r in (8, 16, 32, 64):
+            for M in (8, 64, 256, 1000, 4096, 65536):
+                for k in (1, 8, 16, 32):
+                    if k > M:
+                        continue
+                    p = PX(T, 512, r, M - M % 8 if M >= 8 else 8, k)
+                    assert p.path == mr.PATH_TCGEN05 and p.ctas >= 1
+                    assert p.block_tokens % 32 == 0 and 32 <= p.block_tokens <= 512
