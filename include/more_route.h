@@ -250,14 +250,6 @@ int more_route_status(void* stream);
 /* more_route_launches -- number of kernels this library has launched in this process (all devices). */
 long long more_route_launches(void);
 
-/*
- * more_route_debug_counters -- diagnostic.  Synchronise `stream`, copy the current device's 16 epilogue event
- * counters to out16 (host) and clear them.  The kernels only maintain the counters when the library was built
- * with -DMORE_STATS (chunks, chunks with a hit, triples with a hit, appended candidates, list refreshes, refresh
- * iterations, rescans, element-by-element chunks; the rest unused); otherwise they read zero.
- */
-int more_route_debug_counters(unsigned long long* out16, void* stream);
-
 /* more_strerror -- a static, human-readable string for a MORE_* code. */
 const char* more_strerror(int code);
 

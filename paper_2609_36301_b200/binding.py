@@ -65,6 +65,11 @@ def lib() -> ctypes.CDLL:
         L.more_route_status.restype = i32
         L.more_route_launches.argtypes = []
         L.more_route_launches.restype = ctypes.c_longlong
+        # diagnostics (csrc/more_debug.h; not part of the public interface)
+        L.more_debug_expire_wait.argtypes = [ctypes.c_longlong, vp]
+        L.more_debug_expire_wait.restype = i32
+        L.more_debug_scratch_guard.argtypes = [vp]
+        L.more_debug_scratch_guard.restype = i32
         L.more_strerror.argtypes = [i32]
         L.more_strerror.restype = ctypes.c_char_p
         L.more_version.argtypes = []
@@ -225,6 +230,17 @@ def more_merge_shards(idx, topval, lse, shard_base, M, gate_mode, out_idx, out_g
 
 def more_route_status(stream=None) -> int:
     return int(lib().more_route_status(_stream(stream)))
+
+
+def debug_expire_wait(budget_cycles: int, stream=None) -> int:
+    """Diagnostic: run the library's bounded mbarrier wait on a barrier nobody arrives at, so that it runs out after
+    ``budget_cycles`` clocks and leaves ``MORE_ERR_TIMEOUT`` for :func:`more_route_status` (nothing hangs or faults)."""
+    return int(lib().more_debug_expire_wait(budget_cycles, _stream(stream)))
+
+
+def debug_scratch_guard(stream=None) -> int:
+    """Diagnostic: 1 if the guard region behind the library's scratch allocation is intact, 0 if it was written to."""
+    return int(lib().more_debug_scratch_guard(_stream(stream)))
 
 
 @dataclass

@@ -30,6 +30,7 @@ struct DeviceCtx {
     int sm_count = 0;
     void* scratch = nullptr;
     size_t scratch_bytes = 0;
+    size_t scratch_used = 0;      // bytes the last plan asked for; the guard region starts there
     int* status = nullptr;        // device int: 0 = ok, else a MORE_ERR_* code written by a kernel
     unsigned long long* stats = nullptr;   // 16 diagnostic counters, next to the status word
     void* staging = nullptr;      // device staging of more_route_host

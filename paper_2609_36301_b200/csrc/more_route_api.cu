@@ -1,5 +1,7 @@
 // Host side of libmore_route.so: argument checks, per-device state, launch planning, the extern "C" entry points.
 #include "more_internal.h"
+#include "more_debug.h"
+#include "sm100_common.cuh"
 
 #include <atomic>
 #include <mutex>
@@ -57,6 +59,41 @@ int ensure_bytes(void** buf, size_t* have, size_t need)
     return MORE_OK;
 }
 
+// The scratch allocation always has room for a guard region behind the bytes a plan needs: kGuardBytes of a fixed
+// pattern, written on the caller's stream ahead of the kernels, so that a kernel running past its scratch is caught
+// by more_debug_scratch_guard instead of corrupting whatever lies behind.
+constexpr size_t kGuardBytes = 256;
+constexpr int kGuardPattern = 0x5a;
+
+int ensure_scratch(DeviceCtx* ctx, size_t need, cudaStream_t st)
+{
+    const size_t used = (need + 255) & ~(size_t)255;
+    void* const before = ctx->scratch;
+    int rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, used + kGuardBytes);
+    if (rc != MORE_OK) return rc;
+    if (ctx->scratch != before || used != ctx->scratch_used) {       // (the pattern stays put between calls otherwise)
+        ctx->scratch_used = used;
+        if (cudaMemsetAsync(static_cast<char*>(ctx->scratch) + used, kGuardPattern, kGuardBytes, st) != cudaSuccess)
+            return MORE_ERR_CUDA;
+    }
+    return MORE_OK;
+}
+
+__global__ void expire_wait_kernel(long long budget, int* status)
+{
+    __shared__ uint64_t bar_storage;
+    __shared__ int abort_flag;
+    const uint32_t bar = smem_u32(&bar_storage);
+    if (threadIdx.x == 0) {
+        mbar_init(bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    // nobody arrives: the wait gives up after `budget` clocks, records the time-out and returns false
+    (void)mbar_wait(bar, 0, &abort_flag, status, budget);
+}
+
 int check_shape(int T, int h, int r, int M, int k, int gate_mode, int path)
 {
     if (gate_mode != MORE_GATE_TOPK_SOFTMAX && gate_mode != MORE_GATE_FULL_SOFTMAX) return MORE_ERR_MODE;
@@ -90,7 +127,7 @@ int route_device_locked(const RouteArgs& a, int path, int msplit)
                             ? generic_scratch_bytes(a)
                             : (a.full ? full_scratch_bytes(a, plan)
                                       : (plan.paired ? paired_scratch_bytes(a, plan) : lowrank_scratch_bytes(a, plan)));
-    rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, need);
+    rc = ensure_scratch(ctx, need, a.stream);
     if (rc != MORE_OK) return rc;
     if (a.T == 0 || plan.path != MORE_PATH_TCGEN05) {
         // (the tensor-core launchers clear out_counts themselves, after their last step that can fail)
@@ -370,7 +407,7 @@ int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool fast = fast_ok && path != MORE_PATH_GENERIC;
     if (!fast) {
-        rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, (size_t)T * r * sizeof(float));
+        rc = ensure_scratch(ctx, (size_t)T * r * sizeof(float), st);
         if (rc != MORE_OK) return rc;
     }
     if (cudaMemsetAsync(out_psum, 0, (size_t)M * sizeof(float), st) != cudaSuccess) return MORE_ERR_CUDA;
@@ -395,7 +432,7 @@ int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M
     DeviceCtx* ctx = nullptr;
     int rc = get_ctx(&ctx);
     if (rc != MORE_OK) return rc;
-    rc = ensure_bytes(&ctx->scratch, &ctx->scratch_bytes, dispatch_scratch_bytes(M));
+    rc = ensure_scratch(ctx, dispatch_scratch_bytes(M), static_cast<cudaStream_t>(stream));
     if (rc != MORE_OK) return rc;
     return launch_dispatch(idx, counts, T, k, M, out_offsets, out_sorted_pairs, ctx->scratch,
                            static_cast<cudaStream_t>(stream));
@@ -455,6 +492,35 @@ int more_route_debug_counters(unsigned long long* out16, void* stream)
     if (cudaMemcpyAsync(out16, ctx->stats, 16 * sizeof(unsigned long long), cudaMemcpyDeviceToHost, st) != cudaSuccess) return MORE_ERR_CUDA;
     if (cudaMemsetAsync(ctx->stats, 0, 16 * sizeof(unsigned long long), st) != cudaSuccess) return MORE_ERR_CUDA;
     return cudaStreamSynchronize(st) == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
+
+int more_debug_expire_wait(long long budget_cycles, void* stream)
+{
+    if (budget_cycles < 0 || budget_cycles > 2000000000LL) return MORE_ERR_SHAPE;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    expire_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(budget_cycles, ctx->status);
+    return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
+}
+
+int more_debug_scratch_guard(void* stream)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(&ctx);
+    if (rc != MORE_OK) return rc;
+    if (!ctx->scratch) return 1;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char host[kGuardBytes];
+    if (cudaMemcpyAsync(host, static_cast<char*>(ctx->scratch) + ctx->scratch_used, kGuardBytes, cudaMemcpyDeviceToHost,
+                        st) != cudaSuccess)
+        return MORE_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return MORE_ERR_CUDA;
+    for (size_t i = 0; i < kGuardBytes; ++i)
+        if (host[i] != kGuardPattern) return 0;
+    return 1;
 }
 
 const char* more_strerror(int code)

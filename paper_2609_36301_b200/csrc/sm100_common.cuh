@@ -70,7 +70,8 @@ __device__ __forceinline__ uint32_t mbar_try_wait_now(uint32_t bar, uint32_t par
 }
 
 // Bounded wait.  Returns false if the CTA is aborting (this wait or another one ran out of budget).
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          long long budget = kWaitBudgetCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -78,7 +79,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 15u) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitBudgetCycles) {
+            if (clock64() - t0 > budget) {
                 *abort_flag = 1;
                 atomicExch(status, MORE_ERR_TIMEOUT);
                 return false;

@@ -1,7 +1,12 @@
 """The five benchmark configurations at full size, in the launch configuration the benchmark times (automatic
-path and split).  The oracle is run on a seeded sample of token rows (it computes each row independently);
-properties that hold at any size (counts = bincount of ids, sum = T*k, ids distinct and in range) are checked on
-all rows."""
+path and plan), against the oracle.
+
+c1, c3 and c4 are compared on ALL tokens (the oracle needs 1-15 s per configuration on 16 host cores), every point of
+the expert-count sweep c2 on a contiguous span of 4096 tokens plus the last (ragged) token block.  The histogram must equal the
+oracle's bit for bit once the few exempt near-tie tokens whose sets differ are moved to the experts the GPU chose (for
+c3 that is the benchmark definition's "histogram checked bit-exact").  Properties that hold at any size (counts = bincount of ids, sum = T*k, ids distinct
+and in range, gates summing to 1) are checked on all rows of every configuration.  The exempt-token fraction (oracle
+gap between the k-th and (k+1)-th logit below 1e-3) is printed per configuration."""
 import numpy as np
 import pytest
 
@@ -12,12 +17,11 @@ from helpers import check_rows, to_device
 
 pytestmark = pytest.mark.gpu
 
-SAMPLE_ROWS = 256
-
-CASES = [("c1", 1), ("c1", 0),
-         ("c2_M1024", 0), ("c2_M1024", 1), ("c2_M4096", 0), ("c2_M4096", 1),
-         ("c2_M16384", 0), ("c2_M16384", 1), ("c2_M65536", 0), ("c2_M65536", 1),
-         ("c3", 0), ("c3", 1), ("c4", 1), ("c4", 0)]
+# name, gate mode, rows compared with the oracle (None = all)
+CASES = [("c1", 1, None), ("c1", 0, None),
+         ("c2_M1024", 0, 4096), ("c2_M1024", 1, 4096), ("c2_M4096", 0, 4096), ("c2_M4096", 1, 4096),
+         ("c2_M16384", 0, 4096), ("c2_M16384", 1, 4096), ("c2_M65536", 0, 4096), ("c2_M65536", 1, 4096),
+         ("c3", 0, None), ("c3", 1, None), ("c4", 1, None), ("c4", 0, None)]
 
 _cache = {}
 
@@ -31,8 +35,8 @@ def _case(name):
     return _cache[name]
 
 
-@pytest.mark.parametrize("name,gate_mode", CASES)
-def test_full_config_sampled_rows(name, gate_mode):
+@pytest.mark.parametrize("name,gate_mode,nrows", CASES)
+def test_full_config_against_the_oracle(name, gate_mode, nrows):
     import torch
     case, (X, R1, R2) = _case(name)
     k = case.k
@@ -52,10 +56,51 @@ def test_full_config_sampled_rows(name, gate_mode):
         assert float((gsum - 1).abs().max()) < 1e-5
     else:
         assert float(gsum.max()) <= 1 + 1e-5 and float(res.gate.min()) > 0
-    # sampled rows against the oracle
-    rows = np.sort(np.random.default_rng(1234).choice(case.T, size=SAMPLE_ROWS, replace=False))
-    rt = torch.from_numpy(rows).cuda()
-    st = check_rows(case, rows, res.idx[rt].cpu().numpy(), res.gate[rt].cpu().numpy(), res.topval[rt].cpu().numpy(),
-                    res.lse[rt].cpu().numpy(), gate_mode=gate_mode, k=k)
-    print(f"{name} mode {gate_mode}: exempt {st['exempt']}/{st['tokens']}, differing sets {st['differs']}, "
-          f"gate err {st['gate_err']:.2e}, logit err {st['topval_err']:.2e}, lse err {st['lse_err']:.2e}")
+    # against the oracle
+    if nrows is None:
+        rows = None
+        sel = slice(None)
+    else:
+        # a contiguous span from the middle (several CTAs' worth) plus the last 512 tokens (the final, ragged block)
+        mid = case.T // 2 - nrows // 2
+        rows = np.concatenate([np.arange(mid, mid + nrows), np.arange(case.T - 512, case.T)])
+        sel = torch.from_numpy(rows).cuda()
+    st = check_rows(case, rows, res.idx[sel].cpu().numpy(), res.gate[sel].cpu().numpy(), res.topval[sel].cpu().numpy(),
+                    res.lse[sel].cpu().numpy(), gate_mode=gate_mode, k=k)
+    if nrows is None:
+        # the oracle's histogram, with the (exempt, near-tie) tokens whose sets differ moved to the experts the GPU
+        # chose for them: must equal out_counts bit for bit
+        d = st["differs_mask"]
+        expect = st["ref"].counts.astype(np.int64).copy()
+        if d.any():
+            expect -= np.bincount(st["ref"].idx[d].ravel().astype(np.int64), minlength=case.M)
+            expect += np.bincount(res.idx.cpu().numpy()[d].ravel().astype(np.int64), minlength=case.M)
+        assert np.array_equal(res.counts.cpu().numpy().astype(np.int64), expect), \
+            "out_counts differs from the oracle's histogram"
+    print(f"{name} mode {gate_mode}: {st['tokens']} tokens compared, exempt {st['exempt']} "
+          f"({st['exempt'] / st['tokens']:.2%}), differing sets {st['differs']}, gate err {st['gate_err']:.2e}, "
+          f"logit err {st['topval_err']:.2e}, lse err {st['lse_err']:.2e}"
+          + (", histogram == oracle's" if nrows is None else ""))
+
+
+def test_full_config_top_k_gate_without_extra_outputs():
+    """The launch the benchmark times for the headline configuration: more_route itself (no selected-logit or
+    log-sum-exp outputs, so the kernel variant without the softmax sweep), all tokens against the oracle."""
+    import torch
+    case, (X, R1, R2) = _case("c3")
+    idx = torch.empty((case.T, case.k), dtype=torch.int32, device="cuda")
+    gate = torch.empty((case.T, case.k), dtype=torch.float32, device="cuda")
+    counts = torch.empty((case.M,), dtype=torch.int32, device="cuda")
+    mr.more_route(X, R1, R2, case.k, 0, idx, gate, counts)
+    torch.cuda.synchronize()
+    assert mr.more_route_status() == 0
+    st = check_rows(case, None, idx.cpu().numpy(), gate.cpu().numpy(), gate_mode=0, k=case.k)
+    assert np.array_equal(counts.cpu().numpy().astype(np.int64),
+                          np.bincount(idx.cpu().numpy().ravel().astype(np.int64), minlength=case.M))
+    d = st["differs_mask"]
+    expect = st["ref"].counts.astype(np.int64).copy()
+    if d.any():
+        expect -= np.bincount(st["ref"].idx[d].ravel().astype(np.int64), minlength=case.M)
+        expect += np.bincount(idx.cpu().numpy()[d].ravel().astype(np.int64), minlength=case.M)
+    assert np.array_equal(counts.cpu().numpy().astype(np.int64), expect)
+    print(f"c3 more_route: exempt {st['exempt'] / st['tokens']:.2%}, differing sets {st['differs']}")

@@ -57,3 +57,13 @@ def test_switch_loss_from_counts_and_psum():
     loss_ref = case.M / case.T * float((ref.counts / (case.T * case.k)) @ want)
     assert abs(loss_gpu - loss_ref) <= 1e-3 * loss_ref
     assert loss_ref > 1.2                                                        # a skewed router is far from balanced
+
+
+def test_psum_at_the_benchmarked_size():
+    """c3 at full size (65536 tokens, 16384 experts: the launch the benchmark's psum line times), every bin against
+    the oracle's column sums."""
+    case = inputs.make_config("c3")
+    got, _ = run_psum(case, mr.PATH_AUTO)
+    want, _ = oracle.psum(case.X, case.R1, case.R2)
+    np.testing.assert_allclose(got, want, rtol=RTOL, atol=ATOL)
+    np.testing.assert_allclose(got.sum(), case.T, rtol=1e-4)

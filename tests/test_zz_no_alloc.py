@@ -5,13 +5,15 @@ own pool, or a device allocation would stall their other streams), so ``more_rou
 fixed array inside the library.  That array is shared by all calls and is never cleared, which is exactly what could
 go wrong: this test makes two calls in a row on different problems (the second smaller, so stale contents of the
 first are still lying in the array) and requires each to agree with ``more_route_ex`` on the generic path, which runs
-the same arithmetic out of ordinary scratch.  It lives in a file of its own that is collected last.
+the same arithmetic out of ordinary scratch, and with the CPU oracle.  It lives in a file of its own that is collected last.
 """
 import numpy as np
 import pytest
 
 from paper_2609_36301_b200 import binding as mr
 from paper_2609_36301_b200 import inputs
+
+from helpers import check_counts, check_rows
 
 pytestmark = pytest.mark.gpu
 
@@ -44,6 +46,10 @@ def test_noalloc_matches_ordinary_entry_point_twice_in_a_row():
         assert torch.equal(counts, ref.counts)
         assert float((gate - ref.gate).abs().max()) <= 2e-3             # the tolerance of the parity tests
         assert int(counts.sum()) == case.T * case.k
+        # ... and, in its own right, with the CPU oracle under the acceptance rule of the parity tests
+        st = check_rows(case, None, idx.cpu().numpy(), gate.cpu().numpy(), gate_mode=case.gate_mode, k=case.k)
+        check_counts(idx.cpu().numpy(), counts.cpu().numpy(), case.M, st["ref"].counts,
+                     any_differs=bool(st["differs_mask"].any()))
 
 
 def test_noalloc_rejects_problems_beyond_its_fixed_scratch():
