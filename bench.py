@@ -66,12 +66,18 @@ def roofline(T, h, r, M, k, seconds, peaks, traffic=None):
                 traffic=traffic, peak_source=peaks["source"])
 
 
-# DRAM bytes per launch of route_tcgen05_kernel from ncu captures (dram__bytes_read.sum + dram__bytes_write.sum);
-# the capture behind each figure is summarised under profiles/.  None = not captured for that workload.
-NCU_TRAFFIC_BYTES = {
-    "c3": 274.5e6,          # profiles/route_tcgen05_kernel_c3_ncu_full.md
-    "c2_M16384": 34.78e6,   # profiles/route_tcgen05_kernel_c2_M16384_ncu_full.md
-}
+def load_counters():
+    """Per-workload hardware counters of the router kernel, written when the ncu captures are refreshed: DRAM bytes per
+    launch (dram__bytes_read.sum + dram__bytes_write.sum) and warp instructions per 16-column x 32-token chunk.  A
+    workload that was not captured has no entry."""
+    path = os.path.join(ROOT, "profiles", "counters.json")
+    try:
+        return json.load(open(path))
+    except (OSError, ValueError):
+        return {}
+
+
+SM_COUNT = 148
 
 
 class ClockSampler:
@@ -130,8 +136,10 @@ def describe(name, case, gate_mode):
             f"gate={'full-softmax' if gate_mode else 'topk-softmax'} inputs={case.meta.get('dist')} seed={case.meta.get('seed')}")
 
 
-def oracle_rate(case, gate_mode, target_seconds=12.0):
-    """Tokens/s of the CPU oracle on a bounded prefix sample of the workload's tokens."""
+def oracle_rate(case, gate_mode, target_seconds=25.0):
+    """Tokens/s of the CPU oracle: all tokens of the workload if that fits the time budget (about 11 s for c3 on 16
+    cores), else a bounded prefix; plus the single-thread rate on a 1024-token slice and the exempt-token fraction
+    (oracle gap between the k-th and the (k+1)-th logit below 1e-3) of the sample."""
     import oracle
     probe = min(case.T, 64)
     t0 = time.perf_counter()
@@ -139,9 +147,16 @@ def oracle_rate(case, gate_mode, target_seconds=12.0):
     dt = max(time.perf_counter() - t0, 1e-4)
     n = int(min(case.T, max(probe, probe * target_seconds / dt)))
     t0 = time.perf_counter()
-    oracle.route(case.X[:n], case.R1, case.R2, case.k, gate_mode)
+    ref = oracle.route(case.X[:n], case.R1, case.R2, case.k, gate_mode)
     dt = time.perf_counter() - t0
-    return n / dt, n, dt, oracle.threads()
+    cores = oracle.threads()
+    n1 = min(case.T, 1024)
+    t0 = time.perf_counter()
+    oracle.route(case.X[:n1], case.R1, case.R2, case.k, gate_mode, nthreads=1)
+    dt1 = time.perf_counter() - t0
+    oracle.route(case.X[:8], case.R1, case.R2, case.k, gate_mode, nthreads=cores)    # back to all threads
+    return dict(rate=n / dt, n=n, seconds=dt, cores=cores, single_thread_rate=n1 / dt1,
+                exempt_fraction=float((ref.gap < 1e-3).mean()))
 
 
 def run_reference(args):
@@ -177,6 +192,35 @@ def run_reference(args):
                 cpu_baseline=dict(value=value, unit=UNIT, cores=oracle.threads(), kind="oracle", sample=sample),
                 e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
     print(json.dumps(line))
+
+
+def diagnostic_bounds(T, M, gate_mode, instr_per_chunk, sm_mhz):
+    """What the selection itself costs on the CUDA cores, beside the official roofline: every one of the T*M logits is
+    looked at by a lane.  t_alu: T*M*c lane-operations at 128 lanes per clock and SM, c = the measured warp instructions
+    per 16-column x 32-token chunk / 16 (from the ncu capture; None if the workload was not captured).  t_mufu
+    (full-softmax gate only): T*M exponentials at 16 per clock and SM."""
+    f = (sm_mhz or 1965.0) * 1e6
+    out = dict(t_alu_us=None, lane_ops_per_logit=None, t_mufu_us=None)
+    if instr_per_chunk:
+        c = instr_per_chunk / 16.0
+        out["lane_ops_per_logit"] = c
+        out["t_alu_us"] = T * M * c / (SM_COUNT * 128 * f) * 1e6
+    if gate_mode == 1:
+        out["t_mufu_us"] = T * M / (SM_COUNT * 16 * f) * 1e6
+    return out
+
+
+def host_us_per_call(mr, torch, bufs, k, gate_mode, stream, calls=200):
+    """Host time of one more_route call through the binding (argument checks, plan, descriptor lookup, two enqueues),
+    measured with the stream kept busy so that no call waits for the device."""
+    X, R1, R2, idx, gate, counts = bufs[0]
+    stream.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(calls):
+        mr.more_route(X, R1, R2, k, gate_mode, idx, gate, counts, stream)
+    dt = time.perf_counter() - t0
+    stream.synchronize()
+    return dt / calls * 1e6
 
 
 def time_router(mr, torch, bufs, k, gate_mode, steps, warmup, stream):
@@ -428,17 +472,45 @@ def main():
             dist.destroy_process_group()
         return
 
-    roof = roofline(case.T, case.h, case.r, case.M, k, secs / args.steps, peaks, NCU_TRAFFIC_BYTES.get(name))
-    roof["kernel"] = "route_tcgen05_kernel" if mr.more_route_plan(case.T, case.h, case.r, case.M, k).path == 2 else "generic_route_tokens"
+    counters = load_counters()
+    cnt = counters.get(f"{name}/mode{gate_mode}", {})
+    plan = mr.more_route_plan_ex(case.T, case.h, case.r, case.M, k, gate_mode)
+    roof = roofline(case.T, case.h, case.r, case.M, k, secs / args.steps, peaks, cnt.get("dram_bytes"))
+    roof["kernel"] = ("generic_route_tokens" if plan.path != 2 else
+                      ("route_tcgen05_kernel" if plan.paired else "route_lowrank_kernel"))
+    roof.update(diagnostic_bounds(case.T, case.M, gate_mode, cnt.get("warp_instr_per_chunk"), clocks.get("sm_mhz")))
+    roof["traffic_source"] = cnt.get("source")
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=args.warmup,
                 ms_per_step=secs / args.steps * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16", data="synthetic",
-                config=dict(workload=describe(name, case, gate_mode), l2=l2_note,
-                            plan=vars(mr.more_route_plan(case.T, case.h, case.r, case.M, k))),
+                config=dict(workload=describe(name, case, gate_mode), l2=l2_note, plan=vars(plan)),
                 clocks=clocks, e2e=e2e, gpu_launches=int(launches), roofline=roof)
+
+    # warm-cache time (one copy of the inputs, back to back) beside the cold one; the same thing when X exceeds L2
+    warm = time_router(mr, torch, bufs[:1], k, gate_mode, min(args.steps, 200), 5, stream) / min(args.steps, 200)
+    line["us_cold"] = secs / args.steps * 1e6
+    line["us_warm"] = warm * 1e6
+    line["host_us_per_call"] = host_us_per_call(mr, torch, bufs, k, gate_mode, stream)
+    # routing entropy of the histogram (1 = perfectly balanced), from the last step's out_counts
+    cnts = bufs[0][5].double()
+    pr = cnts / cnts.sum()
+    line["h_norm_counts"] = float(-(pr[pr > 0] * pr[pr > 0].log()).sum() / np.log(case.M))
 
     if not args.no_context:
         extra_entry_points(mr, torch, bufs, case, k, gate_mode, stream, peaks, line)
+        # decode-sized batches: 64 tokens, the expert range cut over the SMs and merged by the last CTA to finish
+        dec = {}
+        for (dh, dr, dM, dk) in ((2048, 64, 16384, 8), (4096, 64, 131072, 16)):
+            dcase = inputs.gaussian_case(64, dh, dr, dM, dk, gate_mode, seed=3)
+            dbufs = make_bufs(torch, dcase, 4)
+            dsecs = time_router(mr, torch, dbufs, dk, gate_mode, 200, 20, stream) / 200
+            dplan = mr.more_route_plan_ex(64, dh, dr, dM, dk, gate_mode)
+            r = roofline(64, dh, dr, dM, dk, dsecs, peaks)
+            dec[f"T=64 h={dh} r={dr} M={dM} k={dk}"] = dict(us=dsecs * 1e6, ctas=dplan.ctas, msplit=dplan.msplit,
+                                                            expert_ranges=dplan.expert_ranges, bound=r["bound"],
+                                                            roofline_frac=r["frac"])
+            del dbufs
+        line["decode"] = dec
 
     # ---- context: unfused library-op router on the same inputs
     ms_unfused = None if args.no_context else unfused_reference_ms(torch, bufs, case, gate_mode)
@@ -446,9 +518,14 @@ def main():
 
     # ---- the CPU oracle on the host cores (a reported baseline, not the target)
     if world == 1 and not args.no_cpu_baseline:
-        rate, n, dt, cores = oracle_rate(case, gate_mode)
-        line["cpu_baseline"] = dict(value=rate, unit=UNIT, cores=cores, kind="oracle",
-                                    sample=f"first {n} of {case.T} tokens of the workload, {dt:.1f} s, fp64 oracle with OpenMP")
+        o = oracle_rate(case, gate_mode)
+        what = "all" if o["n"] == case.T else "first"
+        line["cpu_baseline"] = dict(value=o["rate"], unit=UNIT, cores=o["cores"], kind="oracle",
+                                    sample=f"{what} {o['n']} of {case.T} tokens of the workload, {o['seconds']:.1f} s, "
+                                           "fp64 oracle with OpenMP",
+                                    single_thread_value=o["single_thread_rate"],
+                                    single_thread_sample="first 1024 tokens, one thread")
+        line["exempt_fraction"] = o["exempt_fraction"]
     else:
         line["cpu_baseline"] = None
 
@@ -463,10 +540,17 @@ def main():
                 ocopies, _ = copies_for(ocase)
                 obufs = make_bufs(torch, ocase, ocopies)
                 osecs = time_router(mr, torch, obufs, ocase.k, gm, 200, 50, stream) / 200
+                owarm = time_router(mr, torch, obufs[:1], ocase.k, gm, 200, 5, stream) / 200
                 r = roofline(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k, osecs, peaks)
-                others[f"{oname}/mode{gm}"] = dict(us=osecs * 1e6, tokens_per_s=ocase.T / osecs, bound=r["bound"],
-                                                    roofline_frac=r["frac"],
-                                                    msplit=mr.more_route_plan(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k).msplit)
+                oplan = mr.more_route_plan_ex(ocase.T, ocase.h, ocase.r, ocase.M, ocase.k, gm)
+                ocnt = counters.get(f"{oname}/mode{gm}", {})
+                others[f"{oname}/mode{gm}"] = dict(us=osecs * 1e6, us_warm=owarm * 1e6, tokens_per_s=ocase.T / osecs,
+                                                    bound=r["bound"], roofline_frac=r["frac"], msplit=oplan.msplit,
+                                                    ctas=oplan.ctas, block_tokens=oplan.block_tokens,
+                                                    expert_ranges=oplan.expert_ranges,
+                                                    host_us_per_call=host_us_per_call(mr, torch, obufs, ocase.k, gm, stream, 100),
+                                                    **diagnostic_bounds(ocase.T, ocase.M, gm, ocnt.get("warp_instr_per_chunk"),
+                                                                        clocks.get("sm_mhz")))
                 if oname.startswith("c2_") and not args.no_context:
                     # the expert-count sweep's fused vs unfused-logits comparison (library ops, logits in HBM)
                     ums = unfused_reference_ms(torch, obufs, ocase, gm, iters=3)

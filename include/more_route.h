@@ -231,14 +231,15 @@ int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, 
 /*
  * more_route_plan_ex -- the same report with the whole launch plan of the tensor-core path (Algorithm 1 leaves the
  * block sizes B_N, B_M free; this is how the library chooses them).  want_lse: non-zero if out_lse will be requested.
- *   out7[0] path   out7[1] CTAs per token block   out7[2] total CTAs   out7[3] tokens per CTA
- *   out7[4] 128-token groups per CTA   out7[5] expert ranges swept side by side inside a CTA
- *   out7[6] 1 if the sweep runs on the high half of z and the survivors are rescored in fp32 (top-k-softmax gate
- *           without out_lse, k <= 16, M >= 4096), 0 if every logit is computed from both halves of z
+ *   out8[0] path   out8[1] CTAs per token block   out8[2] total CTAs   out8[3] tokens per CTA
+ *   out8[4] 128-token groups per CTA   out8[5] expert ranges swept side by side inside a CTA
+ *   out8[6] reserved (0)
+ *   out8[7] which of the two kernels: 1 = 256-token CTAs, two per SM, 64-expert steps (many tokens per SM);
+ *           0 = one CTA per SM holding up to four token groups / expert ranges (few tokens per SM)
  * Host-only; needs no device.
  */
 int more_route_plan_ex(int T, int h, int r, int M, int k, int gate_mode, int want_lse, int path, int msplit,
-                       int* out7);
+                       int* out8);
 
 /*
  * more_route_status -- synchronise `stream` and return the sticky device-side status of the current device:

@@ -99,6 +99,7 @@ class RoutePlan:
     token_groups: int = 1
     expert_ranges: int = 1
     filter: bool = False
+    paired: bool = False
 
 
 def more_route_plan(T, h, r, M, k, gate_mode=0, path=PATH_AUTO, msplit=0) -> RoutePlan:
@@ -110,11 +111,11 @@ def more_route_plan(T, h, r, M, k, gate_mode=0, path=PATH_AUTO, msplit=0) -> Rou
 
 
 def more_route_plan_ex(T, h, r, M, k, gate_mode=0, want_lse=False, path=PATH_AUTO, msplit=0) -> RoutePlan:
-    o = (ctypes.c_int * 7)()
+    o = (ctypes.c_int * 8)()
     rc = lib().more_route_plan_ex(T, h, r, M, k, gate_mode, int(want_lse), path, msplit, o)
     if rc != 0:
         raise MoreRouteError(rc, "more_route_plan_ex")
-    return RoutePlan(o[0], o[1], o[2], o[3], o[4], o[5], bool(o[6]))
+    return RoutePlan(o[0], o[1], o[2], o[3], o[4], o[5], bool(o[6]), bool(o[7]))
 
 
 def _ptr(t):

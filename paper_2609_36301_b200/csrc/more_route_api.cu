@@ -439,24 +439,24 @@ int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M
 }
 
 int more_route_plan_ex(int T, int h, int r, int M, int k, int gate_mode, int want_lse, int path, int msplit,
-                       int* out7)
+                       int* out8)
 {
     int rc = check_shape(T, h, r, M, k, gate_mode, path);
     if (rc != MORE_OK) return rc;
-    if (!out7) return MORE_ERR_NULL;
+    if (!out8) return MORE_ERR_NULL;
     Plan p;
     rc = make_plan(T, h, r, M, k, gate_mode, want_lse != 0 || gate_mode == MORE_GATE_FULL_SOFTMAX, false, path, msplit,
                    148, &p);
     if (rc != MORE_OK) return rc;
-    out7[0] = p.path; out7[1] = p.msplit; out7[2] = p.ctas; out7[3] = p.block_tokens;
-    out7[4] = p.tg; out7[5] = p.es; out7[6] = p.filter ? 1 : 0;
+    out8[0] = p.path; out8[1] = p.msplit; out8[2] = p.ctas; out8[3] = p.block_tokens;
+    out8[4] = p.tg; out8[5] = p.es; out8[6] = p.filter ? 1 : 0; out8[7] = p.paired ? 1 : 0;
     return MORE_OK;
 }
 
 int more_route_plan(int T, int h, int r, int M, int k, int gate_mode, int path, int msplit, int* path_out,
                     int* msplit_out, int* ctas_out)
 {
-    int o[7];
+    int o[8];
     const int rc = more_route_plan_ex(T, h, r, M, k, gate_mode, 0, path, msplit, o);
     if (rc != MORE_OK) return rc;
     if (path_out) *path_out = o[0];
