@@ -194,7 +194,13 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
 {
     const int blocks64 = (M + 63) / 64;
     const int rpad = r <= 16 ? 16 : (r <= 32 ? 32 : 64);
-    const bool filter_ok = false;      // (the filter mode is built and tested but is not faster on any measured shape)
+    // The filter mode (sweep on an fp16 rounding of z, exact rescoring of the survivors) is correct but not faster on any
+    // measured shape; it is compiled and planned only in -DMORE_WITH_FILTER builds, which exist to reproduce that.
+#ifdef MORE_WITH_FILTER
+    const bool filter_ok = !want_lse && k <= 16 && M >= 4096;
+#else
+    const bool filter_ok = false;
+#endif
     const double c_lat = want_lse ? 260.0 : 190.0, c_iss = want_lse ? 120.0 : 62.0;
     double best = 1e300;
     Plan bp = *p;

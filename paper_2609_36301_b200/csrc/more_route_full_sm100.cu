@@ -130,7 +130,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
     constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
     using Sel = Selector<KCAP, FILTER, kEpilogueThreads, kCandCap, 4>;
-    constexpr int kCandValStride = Sel::kCandValStride;
+    STAT(constexpr int kCandValStride = Sel::kCandValStride;)
     constexpr int kCandValBytes = Sel::kCandValBytes;
     constexpr int kZoneOff = Sel::kCandBytes;                     // filter: the zone store follows the candidates
     constexpr int kCandBytes = Sel::kCandBytes + (FILTER ? Sel::kZoneBytes : 0);
@@ -850,8 +850,10 @@ int launch_mode(int mode, const CUtensorMap& mx, const CUtensorMap& m1, const CU
 {
     if (mode == 1) return launch_one<RPAD, KCAP, true, FULL, false>(mx, m1, m2, kp, ctas, st, clear_counts);
     if (mode == 0) return launch_one<RPAD, KCAP, false, FULL, false>(mx, m1, m2, kp, ctas, st, clear_counts);
+#ifdef MORE_WITH_FILTER
     if constexpr (!FULL && KCAP <= 16) return launch_one<RPAD, KCAP, false, false, true>(mx, m1, m2, kp, ctas, st, clear_counts);
-    else return MORE_ERR_SHAPE;
+#endif
+    return MORE_ERR_SHAPE;
 }
 
 template <int RPAD, bool FULL>

@@ -78,7 +78,6 @@ constexpr int kBufCols = 32;                       // one accumulator buffer of 
 #endif
 constexpr int kCandCap = MORE_CAND_CAP;            // candidate slots per token
 using SelLayout = Selector<8, true, kEpiThreads, kCandCap, 8>;      // (byte layout only: independent of KCAP, FILTER)
-constexpr int kCandValStride = SelLayout::kCandValStride;
 constexpr int kCandValBytes = SelLayout::kCandValBytes;
 constexpr int kCandBytes = SelLayout::kCandBytes;
 constexpr int kZoneStride = SelLayout::kZoneStride;
@@ -945,8 +944,10 @@ KernelFn kernel_mode(int mode)
         case kModeExact: return kernel_ready<RPAD, KCAP, kModeExact>();
         case kModeExactLse: return kernel_ready<RPAD, KCAP, kModeExactLse>();
         default:
+#ifdef MORE_WITH_FILTER
             if constexpr (KCAP <= 16) return kernel_ready<RPAD, KCAP, kModeFilter>();
-            else return nullptr;
+#endif
+            return nullptr;
     }
 }
 

@@ -25,7 +25,10 @@ static_assert(kStagesP1 * kP1StageBytes <= kRingBytes, "phase-1 ring does not fi
 constexpr int kSmemBytes = kRingBytes + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
 constexpr int kTmemCols = 256;                     // tensor-memory columns per CTA (two CTAs share the 512 of an SM)
 constexpr long long kWaitBudgetCycles = 4000000000LL;   // ~2 s
-constexpr uint32_t kSuspendHintNs = 20000;              // a waiting thread may be parked this long per try
+#ifndef MORE_SUSPEND_NS
+#define MORE_SUSPEND_NS 20000
+#endif
+constexpr uint32_t kSuspendHintNs = MORE_SUSPEND_NS;             // a waiting thread may be parked this long per try
 
 // ------------------------------------------------------------------------------------------------ PTX wrappers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
