@@ -52,7 +52,8 @@ enum {
 enum {
     MORE_OK = 0,
     MORE_ERR_NULL = -1,    /* a required pointer is NULL */
-    MORE_ERR_SHAPE = -2,   /* T < 0; h, r, M or k < 1; k > M; k > MORE_K_MAX; r > MORE_R_MAX; or the forced path cannot run the shape */
+    MORE_ERR_SHAPE = -2,   /* T < 0; h, r, M or k < 1; k > M; k > MORE_K_MAX; r > MORE_R_MAX; M > MORE_M_MAX; msplit outside 0..64;
+                              or the forced path cannot run the shape */
     MORE_ERR_ALIGN = -3,   /* X, R1 or R2 not 16-byte aligned, or an output not 4-byte aligned */
     MORE_ERR_MODE = -4,    /* unknown gate_mode or path */
     MORE_ERR_ARCH = -5,    /* the current device is not compute capability 10.x */
@@ -63,6 +64,7 @@ enum {
 
 #define MORE_K_MAX 32     /* largest k */
 #define MORE_R_MAX 1024   /* largest r (generic path); the tensor-core path takes r <= 64 */
+#define MORE_M_MAX (1 << 30) /* largest M: expert ids, and the kernels' column arithmetic, are 32-bit */
 
 /*
  * more_route -- route T tokens (Algorithm 1 plus the gates of Section 2 / Eq. app_softmax and the per-expert
@@ -89,7 +91,7 @@ int more_route(const void* X, const void* R1, const void* R2,
  *   out_lse     device fp32 [T] or NULL: m_n + log Z_n over all M experts (Eq. app_softmax); computed in either
  *               gate mode when requested (it forces the full-softmax sweep).
  *   path        MORE_PATH_*; a forced path that cannot run the shape gives MORE_ERR_SHAPE.
- *   msplit      tensor-core path only: number of CTAs that share one 256-token block by splitting the expert
+ *   msplit      tensor-core path only: number of CTAs (at most 64) that share one token block by splitting the expert
  *               range (partial top-k lists and (m, Z) pairs are merged by the last CTA to finish);
  *               0 = chosen by the library.  Results do not depend on it.
  */
@@ -221,7 +223,7 @@ int more_dispatch(const int32_t* idx, const int32_t* counts, int T, int k, int M
 /*
  * more_route_plan -- report, without launching, what more_route_ex would do for a shape:
  *   *path_out   MORE_PATH_GENERIC or MORE_PATH_TCGEN05
- *   *msplit_out CTAs per 256-token block (1 on the generic path)
+ *   *msplit_out CTAs per token block (1 on the generic path)
  *   *ctas_out   total CTAs of the main kernel
  * Any of the three may be NULL.  Host-only; needs no device.
  */

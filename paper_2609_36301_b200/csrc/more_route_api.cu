@@ -99,6 +99,7 @@ int check_shape(int T, int h, int r, int M, int k, int gate_mode, int path)
     if (gate_mode != MORE_GATE_TOPK_SOFTMAX && gate_mode != MORE_GATE_FULL_SOFTMAX) return MORE_ERR_MODE;
     if (path != MORE_PATH_AUTO && path != MORE_PATH_GENERIC && path != MORE_PATH_TCGEN05) return MORE_ERR_MODE;
     if (T < 0 || h < 1 || r < 1 || M < 1 || k < 1 || k > M || k > MORE_K_MAX || r > MORE_R_MAX) return MORE_ERR_SHAPE;
+    if (M > MORE_M_MAX) return MORE_ERR_SHAPE;             // expert ids and column counters are 32-bit in the kernels
     return MORE_OK;
 }
 

@@ -43,6 +43,7 @@ def test_bad_arguments_are_rejected_before_any_device_work():
     assert call(T=-1) == -2
     assert call(M=40, k=33) == -2     # k > MORE_K_MAX
     assert call(r=2048) == -2         # r > MORE_R_MAX
+    assert call(M=(1 << 30) + 8) == -2   # M > MORE_M_MAX
     assert call(mode=2) == -4
     assert call(X=None) == -1
     assert call(counts=None) == -1
