@@ -773,23 +773,21 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 epi_sync();
                 if (*last_flag) {
                     __threadfence();
-                    const int64_t base = ((int64_t)blk * p.block_tokens + row_in_blk) * p.msplit;
-                    TopList<KCAP> G;
-                    G.init();
-                    float gm = -INFINITY, gz = 0.f;
-                    if (writer) {
-                        // A token's partial lists lie one after the other in scratch.  Each list's head (its four best
-                        // entries, which is all most lists contribute) is fetched with two 16-byte loads, and the next
-                        // list's head is requested before the current one is merged, so the L2 round trips overlap;
-                        // the tail of a list is read only if its fourth entry still got in.
+                    // Merge of the partial lists [sp_lo, sp_hi) of one token into (G, gm, gz).  A token's lists lie
+                    // one after the other in scratch.  Each list's head (its four best entries, which is all most
+                    // lists contribute) is fetched with two 16-byte loads, and the next list's head is requested
+                    // before the current one is merged, so the L2 round trips overlap; the tail of a list is read
+                    // only if its fourth entry still got in.  Ascending expert ranges: ties keep the smaller id.
+                    auto merge_range = [&](TopList<KCAP>& G, float& gm, float& gz, int tok_in_blk, int sp_lo, int sp_hi) {
+                        const int64_t base = ((int64_t)blk * p.block_tokens + tok_in_blk) * p.msplit;
                         const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
                         const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
-                        float4 hv = __ldcg(pv);
-                        int4 hi = __ldcg(pi);
-                        for (int sp = 0; sp < p.msplit; ++sp) {       // ascending expert ranges: ties keep the smaller id
+                        float4 hv = __ldcg(pv + (size_t)sp_lo * (KCAP / 4));
+                        int4 hi = __ldcg(pi + (size_t)sp_lo * (KCAP / 4));
+                        for (int sp = sp_lo; sp < sp_hi; ++sp) {
                             const float4 cv = hv;
                             const int4 ci = hi;
-                            if (sp + 1 < p.msplit) {
+                            if (sp + 1 < sp_hi) {
                                 hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
                                 hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
                             }
@@ -815,6 +813,52 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                                 gm = nm;
                             }
                         }
+                    };
+                    TopList<KCAP> G;
+                    G.init();
+                    float gm = -INFINITY, gz = 0.f;
+                    // With few tokens and many splits (decode shapes) one thread per token would walk all lists one
+                    // L2 round trip after the other; instead `fan` threads per token merge a contiguous share of the
+                    // ranges each, park their result in the idle ring, and the token's own thread merges those.
+                    int fan = 1;
+                    while (fan < 16 && 2 * fan * p.block_tokens <= kEpiThreads && 4 * fan <= p.msplit) fan *= 2;
+                    if (fan == 1) {
+                        if (writer) merge_range(G, gm, gz, row_in_blk, 0, p.msplit);
+                    } else {
+                        const int bt = p.block_tokens;
+                        float* sv = reinterpret_cast<float*>(ring_ptr);                  // [fan][KCAP][bt]
+                        int* si = reinterpret_cast<int*>(sv + fan * KCAP * bt);         // [fan][KCAP][bt]
+                        float2* smz = reinterpret_cast<float2*>(si + fan * KCAP * bt);  // [fan][bt]
+                        const int wt = etid % bt, wf = etid / bt;
+                        if (wf < fan && wt < live_tokens) {
+                            TopList<KCAP> S;
+                            S.init();
+                            float sm = -INFINITY, sz = 0.f;
+                            merge_range(S, sm, sz, wt, (int)((long long)p.msplit * wf / fan), (int)((long long)p.msplit * (wf + 1) / fan));
+#pragma unroll
+                            for (int s = 0; s < KCAP; ++s) {
+                                sv[(wf * KCAP + s) * bt + wt] = S.v[s];
+                                si[(wf * KCAP + s) * bt + wt] = S.id[s];
+                            }
+                            smz[wf * bt + wt] = make_float2(sm, sz);
+                        }
+                        epi_sync();
+                        if (writer) {
+                            for (int f = 0; f < fan; ++f) {
+                                for (int s = 0; s < KCAP; ++s) {
+                                    const float x = sv[(f * KCAP + s) * bt + row_in_blk];
+                                    if (!(x > G.tau())) break;
+                                    G.insert(x, si[(f * KCAP + s) * bt + row_in_blk]);
+                                }
+                                const float2 mz = smz[f * bt + row_in_blk];
+                                if (LSE && mz.x > -INFINITY) {
+                                    const float nm = fmaxf(gm, mz.x);
+                                    gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
+                                    gm = nm;
+                                }
+                            }
+                        }
+                        epi_sync();                          // the ring is reused by the histogram
                     }
                     hist_clear();
                     if (writer) write_token<KCAP>(p, row, G, gm, gz, hist);
