@@ -188,9 +188,11 @@ void plan_full(int T, int h, int M, int msplit, int sm_count, Plan* p)
 
 // Launch plan of the low-rank router: one CTA per SM with four 128-lane groups, laid out as tg token groups x es expert
 // ranges; msplit CTAs per token block.  A rough cycle model picks among the candidates: a sweep's time per 16-column
-// chunk is the larger of one warp's latency chain and the issue slots of the warps that share a scheduler (one per
-// group), every sweep pays a start-up worth ~160 chunks (nearly every early logit is a candidate), the projection is
-// bounded by the SM's share of HBM bandwidth, and a second wave of CTAs costs a whole CTA time.
+// chunk is the larger of one warp's latency chain and the issue slots of the warps that share a scheduler, every sweep
+// pays a start-up (nearly every early logit is a candidate), the projection is bounded by the SM's share of HBM
+// bandwidth, and a second wave of CTAs costs a whole CTA time.  Measured on B200 the candidates of a small shape lie
+// within ~10 % of each other; what the model must avoid are the outliers (a lone warp sweeping thousands of experts,
+// dozens of partial lists for hundreds of tokens).
 void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, int sm_count, Plan* p)
 {
     const int blocks64 = (M + 63) / 64;
@@ -209,7 +211,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
         const int blocks = (T + bt - 1) / bt;
         const int tg = (bt + 127) / 128;
         for (int es = 1; es * tg <= 4; es *= 2) {
-            if (es > 1 && blocks64 < es * 4) continue;
+            if (blocks64 < es) continue;                       // a range is at least one 64-expert block
             int n1, b1, n2, b2, off;
             if (!lowrank_smem_plan(rpad, tg, es, filter_ok, &n1, &b1, &n2, &b2, &off)) continue;
             int s_lo = 1, s_hi = 1;
@@ -217,7 +219,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
                 s_lo = s_hi = msplit < blocks64 / es ? msplit : (blocks64 / es > 0 ? blocks64 / es : 1);   // at most one CTA per 64-expert block
             } else {
                 s_hi = sm_count / blocks;                      // never more CTAs than one wave
-                if (s_hi > blocks64 / (es * 8)) s_hi = blocks64 / (es * 8);    // a range keeps at least 512 experts
+                if (s_hi > blocks64 / es) s_hi = blocks64 / es;
                 if (s_hi > 64) s_hi = 64;
                 if (s_hi < 1) s_hi = 1;
             }
@@ -225,13 +227,16 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
                 if ((long long)s * es > blocks64) continue;
                 const long long ctas = (long long)blocks * s;
                 const double waves = (double)((ctas + sm_count - 1) / sm_count);
-                const double chunks = 4.0 * blocks64 / (es * s) + 160.0;
+                // a sweep starts with an empty list, so nearly every early logit is a candidate: worth ~160 chunks on a
+                // long range, about ten times its own length on a short one
+                const double range_chunks = 4.0 * ((blocks64 + es * s - 1) / (es * s));     // whole 64-expert steps
+                const double chunks = range_chunks + (range_chunks < 16.0 ? 10.0 * range_chunks : 160.0);
                 const double groups = (double)tg * es;                      // warps per scheduler
                 const double per_chunk = c_lat > groups * c_iss ? c_lat : groups * c_iss;
                 const double ktile = bt * 128.0 / 23.0 > 300.0 ? bt * 128.0 / 23.0 : 300.0;
                 double t = 9000.0 + ((h + 63) / 64) * ktile + chunks * per_chunk;
                 if (es > 1) t += 1500.0;
-                if (s > 1) t += 7000.0 + 60.0 * s;
+                if (s > 1) t += 7000.0 + 60.0 * s + 1.5 * s * bt;      // park, last arriver, its merge of s lists per token
                 const double cost = waves * t;
                 if (cost < best * 0.999) {
                     best = cost;
