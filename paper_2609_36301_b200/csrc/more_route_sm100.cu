@@ -85,6 +85,7 @@ constexpr int kZoneIdOff = SelLayout::kZoneIdOff;
 constexpr int kZoneBytes = SelLayout::kZoneBytes;
 constexpr int kXGroupBytes = 128 * 128;            // X tile of one token group: 128 tokens x 64 bf16
 constexpr int kR1Bytes = 64 * 128;
+constexpr int kMaxStages1 = 8;                     // k-tiles of the projection in flight (a CTA with few tokens is a chain of L2 round trips)
 constexpr int kFallbackSlots = 16;                 // tokens re-routed per round of the fallback (one per epilogue warp)
 constexpr float kLog2e = 1.4426950408889634f;
 
@@ -147,6 +148,185 @@ __device__ __forceinline__ void write_token(const RouteParams& p, int64_t row, c
     if (p.out_lse) p.out_lse[row] = (m2 + log2f(zsum)) * kLn2;
 }
 
+// The CTA that arrives last for a token block merges the partial lists that the block's `msplit` CTAs parked in global
+// scratch: on return the thread of every live token (`writer`, row `row_in_blk` of the block) holds the token's
+// list and (m, Z) pair.  Called by all 512 epilogue threads; the ring (idle by then) is working space.  A function
+// of its own so that its register needs stay out of the sweep's allocation.
+template <int KCAP, bool LSE>
+__device__ __forceinline__ void merge_parked_lists(const RouteParams& p, int blk, int etid, int live_tokens, uint8_t* ring_ptr,
+                                                int row_in_blk, bool writer, TopList<KCAP>& G, float& gm, float& gz)
+{
+    auto epi_sync = [&]() { asm volatile("bar.sync 1, 512;" ::: "memory"); };
+    // Merge of the partial lists [sp_lo, sp_hi) of one token into (G, gm, gz).  A token's lists lie
+    // one after the other in scratch.  Each list's head (its four best entries, which is all most
+    // lists contribute) is fetched with two 16-byte loads, and the next list's head is requested
+    // before the current one is merged, so the L2 round trips overlap; the tail of a list is read
+    // only if its fourth entry still got in.  Ascending expert ranges: ties keep the smaller id.
+    auto merge_range = [&](TopList<KCAP>& G, float& gm, float& gz, int tok_in_blk, int sp_lo, int sp_hi) {
+        const int64_t base = ((int64_t)blk * p.block_tokens + tok_in_blk) * p.msplit;
+        const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
+        const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
+        float4 hv = __ldcg(pv + (size_t)sp_lo * (KCAP / 4));
+        int4 hi = __ldcg(pi + (size_t)sp_lo * (KCAP / 4));
+        for (int sp = sp_lo; sp < sp_hi; ++sp) {
+            const float4 cv = hv;
+            const int4 ci = hi;
+            if (sp + 1 < sp_hi) {
+                hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
+                hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
+            }
+            // each partial list is sorted: stop at the first entry that does not get in
+            bool more = cv.x > G.tau();
+            if (more) G.insert(cv.x, ci.x);
+            more = more && cv.y > G.tau();
+            if (more) G.insert(cv.y, ci.y);
+            more = more && cv.z > G.tau();
+            if (more) G.insert(cv.z, ci.z);
+            more = more && cv.w > G.tau();
+            if (more) G.insert(cv.w, ci.w);
+            for (int s = 4; s < KCAP && more; ++s) {
+                const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
+                const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
+                more = x > G.tau();
+                if (more) G.insert(x, j);
+            }
+            const float2 mz = __ldcg(p.part_mz + base + sp);
+            if (LSE && mz.x > -INFINITY) {
+                const float nm = fmaxf(gm, mz.x);
+                gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
+                gm = nm;
+            }
+        }
+    };
+    G.init();
+    gm = -INFINITY;
+    gz = 0.f;
+    // With few tokens and many splits (decode shapes) one thread per token would walk all lists one
+    // L2 round trip after the other; instead `fan` threads per token merge a contiguous share of the
+    // ranges each, park their result in the idle ring, and the token's own thread merges those.
+    // (Lists of up to 8 entries only: with longer ones this code raises the register needs of the whole kernel, which
+    // costs the sweep of the large k = 16 configurations more than it gains here.)
+    int fan = 1;
+    if constexpr (KCAP <= 8)
+        while (fan < 16 && 2 * fan * p.block_tokens <= kEpiThreads && 4 * fan <= p.msplit) fan *= 2;
+    if (fan == 1) {
+        if (writer) merge_range(G, gm, gz, row_in_blk, 0, p.msplit);
+    } else if constexpr (KCAP <= 8) {
+        // The lists are first copied into the idle ring with coalesced, independent loads (one L2
+        // round trip for all of them instead of one per list and thread), in batches of `lb` lists per
+        // token when they do not fit at once; a token's rows are skewed by 16 bytes against the banks.
+        // All merging is done with the sorted-list network (no data-dependent control flow): a worker
+        // folds its share of the lists into one, then the `fan` lists of a token are merged pairwise
+        // in log2(fan) levels.
+        const int bt = p.block_tokens;
+        constexpr int kPerList = KCAP * 8 + 8;
+    constexpr int kInFlight = 4;                          // loads per array and thread in flight during the copy
+        float* sv = reinterpret_cast<float*>(ring_ptr);                  // [fan][KCAP][bt]
+        int* si = reinterpret_cast<int*>(sv + fan * KCAP * bt);         // [fan][KCAP][bt]
+        float2* smz = reinterpret_cast<float2*>(si + fan * KCAP * bt);  // [fan][bt]
+        const int sub_bytes = (fan * bt * kPerList + 127) & ~127;
+        int lb = ((kRRing - sub_bytes) / bt - 40) / kPerList;
+        lb = lb < p.msplit ? lb : p.msplit;
+        const int tsv = lb * KCAP + 4, tsm = lb + 1;        // a token's stride in floats / in float2s
+        float* av = reinterpret_cast<float*>(ring_ptr + sub_bytes);      // [bt][lb][KCAP] (+ skew)
+        int* ai = reinterpret_cast<int*>(av + bt * tsv);
+        float2* amz = reinterpret_cast<float2*>(ai + bt * tsv);
+        const int wt = etid % bt, wf = etid / bt;
+        const bool worker = wf < fan && wt < live_tokens;
+        const int share_lo = (int)((long long)p.msplit * wf / fan), share_hi = (int)((long long)p.msplit * (wf + 1) / fan);
+        TopList<KCAP> S;
+        S.init();
+        float sm = -INFINITY, sz = 0.f;
+        auto join_mz = [&](const float2 mz) {
+            if (LSE && mz.x > -INFINITY) {
+                const float nm = fmaxf(sm, mz.x);
+                sz = sz * ex2f(sm - nm) + mz.y * ex2f(mz.x - nm);
+                sm = nm;
+            }
+        };
+        const int64_t blk_slot = (int64_t)blk * bt * p.msplit;
+        const float4* gv = reinterpret_cast<const float4*>(p.part_val);
+        const int4* gi = reinterpret_cast<const int4*>(p.part_id);
+        for (int sp0 = 0; sp0 < p.msplit; sp0 += lb) {
+            const int nl = min(lb, p.msplit - sp0);
+            const int q4 = nl * (KCAP / 4);
+            const int total = live_tokens * q4;
+            for (int e0 = etid; e0 < total; e0 += kInFlight * kEpiThreads) {
+                float4 xv[kInFlight];
+                int4 xi[kInFlight];
+                int dst[kInFlight];
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) {
+                    const int e = e0 + u * kEpiThreads;
+                    dst[u] = -1;
+                    if (e < total) {
+                        const int t = e / q4, w = e - t * q4;
+                        const int64_t src = (blk_slot + (int64_t)t * p.msplit + sp0) * (KCAP / 4) + w;
+                        xv[u] = __ldcg(gv + src);
+                        xi[u] = __ldcg(gi + src);
+                        dst[u] = t * (tsv / 4) + w;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) {
+                    if (dst[u] >= 0) {
+                        reinterpret_cast<float4*>(av)[dst[u]] = xv[u];
+                        reinterpret_cast<int4*>(ai)[dst[u]] = xi[u];
+                    }
+                }
+            }
+            if (LSE) {
+                for (int e = etid; e < live_tokens * nl; e += kEpiThreads) {
+                    const int t = e / nl, l = e - t * nl;
+                    amz[t * tsm + l] = __ldcg(p.part_mz + blk_slot + (int64_t)t * p.msplit + sp0 + l);
+                }
+            }
+            epi_sync();
+            if (worker) {
+                const int lo = max(share_lo, sp0), hi = min(share_hi, sp0 + nl);
+                for (int sp = lo; sp < hi; ++sp) {
+                    const float* lv = av + wt * tsv + (sp - sp0) * KCAP;
+                    const int* li = ai + wt * tsv + (sp - sp0) * KCAP;
+                    S.merge_sorted([&](int e) { return lv[e]; }, [&](int e) { return li[e]; });
+                    if (LSE) join_mz(amz[wt * tsm + (sp - sp0)]);
+                }
+            }
+            epi_sync();
+        }
+        auto park_sub = [&]() {
+#pragma unroll
+            for (int s = 0; s < KCAP; ++s) {
+                sv[(wf * KCAP + s) * bt + wt] = S.v[s];
+                si[(wf * KCAP + s) * bt + wt] = S.id[s];
+            }
+            smz[wf * bt + wt] = make_float2(sm, sz);
+        };
+        if (worker) park_sub();
+        epi_sync();
+        for (int d = 1; d < fan; d <<= 1) {
+            if (worker && (wf & (2 * d - 1)) == 0) {
+                S.merge_sorted([&](int e) { return sv[((wf + d) * KCAP + e) * bt + wt]; },
+                               [&](int e) { return si[((wf + d) * KCAP + e) * bt + wt]; });
+                if (LSE) join_mz(smz[(wf + d) * bt + wt]);
+                if (2 * d < fan) park_sub();
+                else if (wf == 0) park_sub();
+            }
+            epi_sync();
+        }
+        if (writer) {
+#pragma unroll
+            for (int s = 0; s < KCAP; ++s) {
+                G.v[s] = sv[s * bt + row_in_blk];
+                G.id[s] = si[s * bt + row_in_blk];
+            }
+            const float2 mz = smz[row_in_blk];
+            gm = mz.x;
+            gz = mz.y;
+        }
+        epi_sync();                          // the ring is reused by the histogram
+    }
+}
+
 // ------------------------------------------------------------------------------------------------- the kernel
 template <int RPAD, int KCAP, int MODE>
 __global__ void __launch_bounds__(kRThreads, 1)
@@ -169,7 +349,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     uint8_t* ring_ptr = smem_raw + (ring - raw);
     uint8_t* ctl = ring_ptr + kRRing;                        // control block
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
-    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + 4, B_ZACC = B_EMPTY1 + 4, B_FULL2 = B_ZACC + 1,
+    constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kMaxStages1, B_ZACC = B_EMPTY1 + kMaxStages1, B_FULL2 = B_ZACC + 1,
                   B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_COUNT = B_ACCF + kGroups * 3;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
@@ -202,7 +382,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int e = 0; e < es; ++e) part_tab[e] = (int)(((long long)p.blocks64 * (split * es + e)) / nparts);
-        for (int i = 0; i < 4; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
+        for (int i = 0; i < kMaxStages1; ++i) { mbar_init(bar(B_FULL1 + i), 1); mbar_init(bar(B_EMPTY1 + i), 1); }
         mbar_init(bar(B_ZACC), 1);
         // a stage is free again when both 32-expert halves of every group's step have been multiplied
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 2 * ngroups); }
@@ -732,7 +912,8 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // memory and flushes only the non-zero bins with one global atomic each; otherwise straight to global memory
         // (with that many experts the bins hardly collide).  With few experts thousands of pairs hit each bin, and
         // same-address global atomics would serialise.
-        int* hist = (p.M <= kRRing / 4) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
+        // (a CTA with few tokens would spend longer clearing and flushing the bins than on its handful of atomics)
+        int* hist = (p.M <= kRRing / 4 && live_tokens * p.k * 16 > p.M) ? reinterpret_cast<int*>(ring_ptr) : nullptr;
         auto hist_clear = [&]() {
             if (hist) {
                 for (int e = etid; e < p.M; e += kEpiThreads) hist[e] = 0;
@@ -773,93 +954,9 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 epi_sync();
                 if (*last_flag) {
                     __threadfence();
-                    // Merge of the partial lists [sp_lo, sp_hi) of one token into (G, gm, gz).  A token's lists lie
-                    // one after the other in scratch.  Each list's head (its four best entries, which is all most
-                    // lists contribute) is fetched with two 16-byte loads, and the next list's head is requested
-                    // before the current one is merged, so the L2 round trips overlap; the tail of a list is read
-                    // only if its fourth entry still got in.  Ascending expert ranges: ties keep the smaller id.
-                    auto merge_range = [&](TopList<KCAP>& G, float& gm, float& gz, int tok_in_blk, int sp_lo, int sp_hi) {
-                        const int64_t base = ((int64_t)blk * p.block_tokens + tok_in_blk) * p.msplit;
-                        const float4* pv = reinterpret_cast<const float4*>(p.part_val + base * KCAP);
-                        const int4* pi = reinterpret_cast<const int4*>(p.part_id + base * KCAP);
-                        float4 hv = __ldcg(pv + (size_t)sp_lo * (KCAP / 4));
-                        int4 hi = __ldcg(pi + (size_t)sp_lo * (KCAP / 4));
-                        for (int sp = sp_lo; sp < sp_hi; ++sp) {
-                            const float4 cv = hv;
-                            const int4 ci = hi;
-                            if (sp + 1 < sp_hi) {
-                                hv = __ldcg(pv + (size_t)(sp + 1) * (KCAP / 4));
-                                hi = __ldcg(pi + (size_t)(sp + 1) * (KCAP / 4));
-                            }
-                            // each partial list is sorted: stop at the first entry that does not get in
-                            bool more = cv.x > G.tau();
-                            if (more) G.insert(cv.x, ci.x);
-                            more = more && cv.y > G.tau();
-                            if (more) G.insert(cv.y, ci.y);
-                            more = more && cv.z > G.tau();
-                            if (more) G.insert(cv.z, ci.z);
-                            more = more && cv.w > G.tau();
-                            if (more) G.insert(cv.w, ci.w);
-                            for (int s = 4; s < KCAP && more; ++s) {
-                                const float x = __ldcg(p.part_val + (base + sp) * KCAP + s);
-                                const int j = __ldcg(p.part_id + (base + sp) * KCAP + s);
-                                more = x > G.tau();
-                                if (more) G.insert(x, j);
-                            }
-                            const float2 mz = __ldcg(p.part_mz + base + sp);
-                            if (LSE && mz.x > -INFINITY) {
-                                const float nm = fmaxf(gm, mz.x);
-                                gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
-                                gm = nm;
-                            }
-                        }
-                    };
                     TopList<KCAP> G;
-                    G.init();
-                    float gm = -INFINITY, gz = 0.f;
-                    // With few tokens and many splits (decode shapes) one thread per token would walk all lists one
-                    // L2 round trip after the other; instead `fan` threads per token merge a contiguous share of the
-                    // ranges each, park their result in the idle ring, and the token's own thread merges those.
-                    int fan = 1;
-                    while (fan < 16 && 2 * fan * p.block_tokens <= kEpiThreads && 4 * fan <= p.msplit) fan *= 2;
-                    if (fan == 1) {
-                        if (writer) merge_range(G, gm, gz, row_in_blk, 0, p.msplit);
-                    } else {
-                        const int bt = p.block_tokens;
-                        float* sv = reinterpret_cast<float*>(ring_ptr);                  // [fan][KCAP][bt]
-                        int* si = reinterpret_cast<int*>(sv + fan * KCAP * bt);         // [fan][KCAP][bt]
-                        float2* smz = reinterpret_cast<float2*>(si + fan * KCAP * bt);  // [fan][bt]
-                        const int wt = etid % bt, wf = etid / bt;
-                        if (wf < fan && wt < live_tokens) {
-                            TopList<KCAP> S;
-                            S.init();
-                            float sm = -INFINITY, sz = 0.f;
-                            merge_range(S, sm, sz, wt, (int)((long long)p.msplit * wf / fan), (int)((long long)p.msplit * (wf + 1) / fan));
-#pragma unroll
-                            for (int s = 0; s < KCAP; ++s) {
-                                sv[(wf * KCAP + s) * bt + wt] = S.v[s];
-                                si[(wf * KCAP + s) * bt + wt] = S.id[s];
-                            }
-                            smz[wf * bt + wt] = make_float2(sm, sz);
-                        }
-                        epi_sync();
-                        if (writer) {
-                            for (int f = 0; f < fan; ++f) {
-                                for (int s = 0; s < KCAP; ++s) {
-                                    const float x = sv[(f * KCAP + s) * bt + row_in_blk];
-                                    if (!(x > G.tau())) break;
-                                    G.insert(x, si[(f * KCAP + s) * bt + row_in_blk]);
-                                }
-                                const float2 mz = smz[f * bt + row_in_blk];
-                                if (LSE && mz.x > -INFINITY) {
-                                    const float nm = fmaxf(gm, mz.x);
-                                    gz = gz * ex2f(gm - nm) + mz.y * ex2f(mz.x - nm);
-                                    gm = nm;
-                                }
-                            }
-                        }
-                        epi_sync();                          // the ring is reused by the histogram
-                    }
+                    float gm, gz;
+                    merge_parked_lists<KCAP, LSE>(p, blk, etid, live_tokens, ring_ptr, row_in_blk, writer, G, gm, gz);
                     hist_clear();
                     if (writer) write_token<KCAP>(p, row, G, gm, gz, hist);
                     hist_flush();
@@ -1059,7 +1156,7 @@ bool lowrank_smem_plan(int rpad, int tg, int es, bool filter, int* nst1, int* st
     if (n2 == 3) n2 = 2;
     const int off = (kRRing - n2 * st2) & ~1023;
     int n1 = off / st1;
-    if (n1 > 4) n1 = 4;
+    if (n1 > kMaxStages1) n1 = kMaxStages1;
     if (n1 < 1) return false;
     *nst1 = n1; *st1_bytes = st1; *nst2 = n2; *st2_bytes = st2; *r2_off = off;
     return true;

@@ -42,6 +42,35 @@ struct TopList {
         v[0] = top ? x : v[0];
         id[0] = top ? j : id[0];
     }
+    // Replace this list by the KCAP best of it and of another sorted list under the full order (value descending, id
+    // ascending); other_v(s) / other_id(s) return entry s of the other list (read where it lies: no second list in
+    // registers).  Entry s against the other list's entry KCAP-1-s keeps the KCAP best of the union as a bitonic
+    // sequence, which log2(KCAP) stages of compare-exchanges sort: straight-line code, the same work whatever the data.
+    template <class FV, class FI>
+    __device__ __forceinline__ void merge_sorted(FV other_v, FI other_id)
+    {
+#pragma unroll
+        for (int s = 0; s < KCAP; ++s) {
+            const float x = other_v(KCAP - 1 - s);
+            const int j = other_id(KCAP - 1 - s);
+            const bool take = x > v[s] || (x == v[s] && j < id[s]);
+            v[s] = take ? x : v[s];
+            id[s] = take ? j : id[s];
+        }
+#pragma unroll
+        for (int stride = KCAP / 2; stride > 0; stride >>= 1) {
+#pragma unroll
+            for (int s = 0; s < KCAP; ++s) {
+                if ((s & stride) == 0) {
+                    const int t = s + stride;
+                    const bool swap = v[t] > v[s] || (v[t] == v[s] && id[t] < id[s]);
+                    const float hv = swap ? v[t] : v[s], lv = swap ? v[s] : v[t];
+                    const int hi = swap ? id[t] : id[s], li = swap ? id[s] : id[t];
+                    v[s] = hv; v[t] = lv; id[s] = hi; id[t] = li;
+                }
+            }
+        }
+    }
     // Insert with the full order (value descending, id ascending): for merging lists whose ids interleave.
     __device__ __forceinline__ void insert_ordered(float x, int j)
     {
