@@ -231,7 +231,11 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
                 // long range, about ten times its own length on a short one
                 const double range_chunks = 4.0 * ((blocks64 + es * s - 1) / (es * s));     // whole 64-expert steps
                 const double chunks = range_chunks + (range_chunks < 16.0 ? 10.0 * range_chunks : 160.0);
-                const double groups = (double)tg * es;                      // warps per scheduler
+                // warps per scheduler: one per group, except that a block of at most 64 tokens is spread over the
+                // lane quarters, one or two quarters per expert range (credited only to small problems: on long
+                // sweeps the latency term of this model is too optimistic for two warps per scheduler)
+                double groups = (double)tg * es;
+                if (tg == 1 && bt <= 64 && es >= 2 && blocks * 8 <= sm_count) groups = bt <= 32 ? 1.0 : (es == 4 ? 2.0 : 1.0);
                 const double per_chunk = c_lat > groups * c_iss ? c_lat : groups * c_iss;
                 const double ktile = bt * 128.0 / 23.0 > 300.0 ? bt * 128.0 / 23.0 : 300.0;
                 double t = 9000.0 + ((h + 63) / 64) * ktile + chunks * per_chunk;

@@ -94,6 +94,7 @@ enum { kModeExact = 0, kModeExactLse = 1, kModeFilter = 2 };
 struct RouteParams {
     int T, h, r, M, k, gate_mode;
     int msplit, es, tg;          // CTAs per token block; expert ranges and token groups inside a CTA
+    int spread;                  // a block of at most 64 tokens is repeated over the 128 tensor-memory lanes (see the kernel)
     int block_tokens;            // tokens per CTA: a multiple of 32, at most 128 * tg
     int blocks64;                // ceil(M / 64)
     int nst1, st1_bytes;         // phase-1 stages
@@ -416,8 +417,14 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 if (!ok) break;
                 const uint32_t dst = ring + s * p.st1_bytes;
                 mbar_expect_tx(bar(B_FULL1 + s), st1_tx);
-                for (int t = 0; t < tg_live; ++t)                   // 128 token rows x 64 columns per token group
-                    tma_load_2d(dst + t * kXGroupBytes, &map_x, bar(B_FULL1 + s), kt * 64, tok0 + t * 128);
+                if (p.spread) {                                     // 4 x (32 token rows x 64 columns): the block, repeated
+                    for (int j = 0; j < 4; ++j)
+                        tma_load_2d(dst + j * (kXGroupBytes / 4), &map_x, bar(B_FULL1 + s), kt * 64,
+                                    tok0 + (j * 32) % p.block_tokens);
+                } else {
+                    for (int t = 0; t < tg_live; ++t)               // 128 token rows x 64 columns per token group
+                        tma_load_2d(dst + t * kXGroupBytes, &map_x, bar(B_FULL1 + s), kt * 64, tok0 + t * 128);
+                }
                 tma_load_2d(dst + p.tg * kXGroupBytes, &map_r1, bar(B_FULL1 + s), 0, kt * 64);
             }
             // the R2 stages lie beyond the phase-1 stages, so the first blocks of R2 arrive while phase 1 still runs
@@ -463,10 +470,16 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int q = warp & 3;                              // TMEM lane quarter this warp may access
         const int etid = threadIdx.x - 32 * kFirstEpiWarp;   // 0..511 among the epilogue threads
         const int tgi = g / es, esi = g % es;
-        const int row_in_tg = q * 32 + lane;
+        // Which token a lane holds.  Normally lane quarter q of token group tgi holds tokens tgi*128 + q*32 ...  A block
+        // of at most 64 tokens (p.spread) is instead loaded into every 32- or 64-lane stretch of the group's 128 lanes,
+        // so all stretches hold the same z, and expert range esi works on stretch esi: the few working warps of such a
+        // CTA then sit in different lane quarters, i.e. on different schedulers, instead of all on the first one or two.
+        const int lq = p.block_tokens >> 5;                                   // spread: lane quarters per copy (1 or 2)
+        const int qi = p.spread ? ((q - esi * lq) & 3) : q;                  // this warp's index in its group's stretch
+        const int row_in_tg = qi * 32 + lane;
         const int row_in_blk = tgi * 128 + row_in_tg;
         const int64_t row = (int64_t)tok0 + row_in_blk;
-        const bool warp_live = g < ngroups && (tgi * 128 + q * 32) < live_tokens;     // warp-uniform
+        const bool warp_live = g < ngroups && (tgi * 128 + qi * 32) < live_tokens && (!p.spread || qi < lq);     // warp-uniform
         const bool row_live = warp_live && row_in_blk < live_tokens;
         const uint32_t t_lanes = tmem_base + ((uint32_t)(q * 32) << 16);
         const uint32_t t_zacc = t_lanes + (tgi * es) * kGroupCols + kRingCol0;       // the token group's z (fp32)
@@ -629,10 +642,16 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
             S.scan(v, t, col0);
         };
         // ---- after the two chunks of a buffer: fold if some token of the warp could overflow on the next buffer
-        auto fold_check = [&]() {
+        // (the first two buffers of a sweep are folded wholesale: with a near-empty list almost everything gets in)
+        auto fold_check = [&](int n) {
             if (__any_sync(kFullMask, S.ptr >= S.warn)) {
                 STAT(st_fold++; const long long tr0 = clock64();)
-                S.fold();
+                if constexpr (FILTER) {
+                    S.fold();
+                } else {
+                    if (n < 2) S.fold_all();
+                    else S.fold();
+                }
                 STAT(st_tfold += clock64() - tr0;)
             }
         };
@@ -647,7 +666,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         // group would exceed the thread count that leaves 96 registers per thread.)
         if (nb > 0 && ok) {
             int slot = 0, pslot = 0, all_out = lw;                 // `released` reads all_out once every warp is out
-            int my_refill = q + 1;                                 // next iteration at which this warp refills a slot
+            int my_refill = qi + 1;                                // next iteration at which this warp refills a slot
             uint32_t ph = 0;
             const uint32_t rel0 = smem_u32(released + g * 3);
             // One iteration = one buffer.  `masked` (a compile-time flag, so that the common iterations carry none of
@@ -705,7 +724,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         if (col0 + 16 + i >= e_hi) vb[i] = -INFINITY;
                 }
                 process(vb, col0 + 16);
-                fold_check();
+                fold_check(n);
                 pslot = slot;
                 if (++slot == NBUF) { slot = 0; ph ^= 1; all_out += lw; }
             };
@@ -1181,7 +1200,9 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     const ScratchLayout L = scratch_layout(a, p);
     char* base = static_cast<char*>(scratch);
     CUtensorMap mx, m1, m2;
-    int rc = get_tensor_map(a.X, a.T, a.h, 128, 64, &mx);
+    // few tokens and several expert ranges per CTA: spread the working warps over the lane quarters (see the kernel)
+    const bool spread = p.tg == 1 && p.block_tokens <= 64 && p.es >= 2;
+    int rc = get_tensor_map(a.X, a.T, a.h, spread ? 32 : 128, 64, &mx);
     if (rc == MORE_OK) rc = get_tensor_map(a.R1, a.h, a.r, 64, 64, &m1);
     // the filter sweeps the fp16 copy of R2 in scratch (same shape; a 16-bit type either way as far as TMA cares)
     if (rc == MORE_OK) rc = get_tensor_map(p.filter ? static_cast<const void*>(base + L.r2h) : a.R2, a.r, a.M, rpad, 64, &m2);
@@ -1189,6 +1210,7 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
 
     rp.T = a.T; rp.h = a.h; rp.r = a.r; rp.M = a.M; rp.k = a.k; rp.gate_mode = a.gate_mode;
     rp.msplit = p.msplit; rp.es = p.es; rp.tg = p.tg;
+    rp.spread = spread ? 1 : 0;
     rp.block_tokens = p.block_tokens;
     rp.blocks64 = (a.M + 63) / 64;
     rp.out_idx = a.out_idx; rp.out_gate = a.out_gate; rp.out_counts = a.out_counts;

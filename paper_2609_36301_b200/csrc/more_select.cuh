@@ -223,6 +223,31 @@ struct Selector {
         cptr = cbase;
         thr = limit();
     }
+    // The same result as fold() for the start of a sweep, when nearly every buffered element still gets in: every
+    // element of every entry is offered to the list in column order (an insert changes nothing for a value at or
+    // below the list's last), straight-line code instead of one data-dependent round per element.  Not for FILTER.
+    __device__ __forceinline__ void fold_all()
+    {
+        static_assert(!FILTER, "the zone store needs fold()");
+        uint32_t a = base, c = cbase;
+        while (__any_sync(kFullMask, a < ptr)) {
+            float x0 = -INFINITY, x1 = -INFINITY, x2 = -INFINITY, x3 = -INFINITY;
+            int col = 0;
+            if (a < ptr) {
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=f"(x0), "=f"(x1), "=f"(x2), "=f"(x3) : "r"(a) : "memory");
+                col = lds_s32(c);
+            }
+            L.insert(x0, col);
+            L.insert(x1, col + 1);
+            L.insert(x2, col + 2);
+            L.insert(x3, col + 3);
+            a += kCandValStride;
+            c += kCandColStride;
+        }
+        ptr = base;
+        cptr = cbase;
+        thr = limit();
+    }
     // if (t > thr) append {v0, v1, v2, v3} and col
     __device__ __forceinline__ void append4(float t, float v0, float v1, float v2, float v3, int col)
     {
