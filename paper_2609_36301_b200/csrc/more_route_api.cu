@@ -152,8 +152,8 @@ void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 
 namespace {
 
-// Launch plan of the fused standard router (256-token CTAs, two per SM).
-void plan_full(int T, int h, int M, int msplit, int sm_count, Plan* p)
+// Launch plan of the paired low-rank kernel (256-token CTAs, two per SM).
+void plan_paired(int T, int h, int M, int msplit, int sm_count, Plan* p)
 {
     const int slots = 2 * sm_count;                       // two CTAs are resident per SM
     const int tiles = (M + kTileExperts - 1) / kTileExperts;
@@ -180,6 +180,36 @@ void plan_full(int T, int h, int M, int msplit, int sm_count, Plan* p)
         const double per_cta = 256.0 * (h / 8.0) + (double)bt * ((double)tiles / s) * 16.0 + 256.0 * 256.0;
         const double cost = per_sm * per_cta;
         if (cost < best * 0.999) { best = cost; best_bt = bt; best_s = s; }
+    }
+    p->block_tokens = best_bt;
+    p->msplit = best_s;
+    p->ctas = ((T + best_bt - 1) / best_bt) * best_s;
+}
+
+// Launch plan of the fused standard router: one CTA per SM, 256-expert steps that each run over all h/64 k-tiles.  A
+// step costs the same whatever the block's fill (the MMAs are 128 tokens tall regardless), so what counts is waves x
+// steps per CTA; splitting the experts over a few CTAs per token block evens out the last wave.
+void plan_dense(int T, int h, int M, int msplit, int sm_count, Plan* p)
+{
+    const int tiles = (M + 255) / 256;
+    const double ktiles = (h + 63) / 64;
+    double best = 1e300;
+    int best_bt = kBlockTokens, best_s = 1;
+    for (int bt = kBlockTokens; bt >= 128; bt -= 32) {
+        const int blocks = (T + bt - 1) / bt;
+        const int s_lo = msplit > 0 ? (msplit < tiles ? msplit : tiles) : 1;
+        const int s_hi = msplit > 0 ? s_lo : (tiles < 16 ? tiles : 16);
+        for (int s = s_lo; s <= s_hi; ++s) {
+            const long long ctas = (long long)blocks * s;
+            const double waves = (double)((ctas + sm_count - 1) / sm_count);
+            const double steps = (double)((tiles + s - 1) / s);
+            // microseconds, fitted to B200 measurements: 1.2 per k-tile of a step (the L2 -> SM traffic of the
+            // stages), 2.1 for its epilogue, 8 per CTA for start and pipeline fill, 25 more when the lists are
+            // parked and merged
+            double cost = waves * (steps * (1.2 * ktiles + 2.1) + 8.0 + (s > 1 ? 25.0 : 0.0));
+            cost *= 1.0 + 0.02 * (kBlockTokens - bt) / 32.0;          // prefer full blocks on a tie
+            if (cost < best * 0.999) { best = cost; best_bt = bt; best_s = s; }
+        }
     }
     p->block_tokens = best_bt;
     p->msplit = best_s;
@@ -275,7 +305,7 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
     p.path = MORE_PATH_TCGEN05;
     if (sm_count <= 0) sm_count = 148;
     if (full) {
-        plan_full(T, h, M, msplit, sm_count, &p);
+        plan_dense(T, h, M, msplit, sm_count, &p);
     } else {
         // Two kernels serve the low-rank router (measured on B200, both gate modes, T from 8 k to 64 k tokens): the
         // grouped kernel (one CTA per SM, up to four token groups / expert ranges side by side) wins while an SM has
@@ -290,7 +320,7 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
         if (grouped) {
             plan_lowrank(T, h, r, M, k, want_lse, msplit, sm_count, &p);
         } else {
-            plan_full(T, h, M, msplit, sm_count, &p);
+            plan_paired(T, h, M, msplit, sm_count, &p);
             p.paired = true;
         }
         if (p.block_tokens == 0) return MORE_ERR_SHAPE;

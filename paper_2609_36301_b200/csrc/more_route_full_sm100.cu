@@ -50,6 +50,8 @@ namespace {
 #ifndef MORE_CAND_CAP
 #define MORE_CAND_CAP 8
 #endif
+// fused standard router: three stages of (256 x 64 X tile + 64 x 256 W tile) and six candidate slots per token
+constexpr int kFullRingBytes = 3 * (kXTileBytes + 4 * 64 * 128) + 6 * kEpilogueThreads * 20;
 constexpr int kFallbackSlots = 8;      // tokens re-routed per round of the filter's fallback (one per epilogue warp)
 
 struct KernelParams {
@@ -110,9 +112,11 @@ __device__ __forceinline__ void write_token(const KernelParams& p, int64_t row, 
 
 // ------------------------------------------------------------------------------------------------- the kernel
 // FULL = true is the fused STANDARD router (logits = X W with W [h][M], no low-rank bottleneck: Alg. 1 without z, the
-// contraction running over K = h): there is no phase 1, every 64-expert step instead accumulates over all h/64 k-tiles
-// of X (256 x 64, re-read per step) and W (64 x 64) with the phase-1 pipeline and stage layout, and the epilogue is
-// the same.  map_r2 is then W's map (64 x 64 boxes), map_r1 is unused, RPAD is 64.
+// contraction running over K = h): there is no phase 1; every step accumulates 256 experts over all h/64 k-tiles of X
+// (256 x 64) and W (64 x 256, four 64 x 64 boxes), so X is re-read from L2 once per 256 experts.  That takes all 512
+// tensor-memory columns (two 128-token x 256-expert accumulators) and three 64 KB stages: one CTA per SM.  The epilogue
+// is the same, run over four 64-column quarters per step.  map_r2 is then W's map (64 x 64 boxes), map_r1 is unused,
+// RPAD is 64.
 //
 // FILTER = true (low-rank router, top-k-softmax gate, no log-sum-exp): the second contraction runs on one fp16 rounding
 // of z (scaled per token by a power of two) against an fp16 copy of R2, i.e. half the MMAs; the selection keeps every
@@ -125,7 +129,11 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                      const __grid_constant__ CUtensorMap map_r2, const KernelParams p)
 {
     constexpr int kKSteps = RPAD / 16;                          // UMMA K = 16
-    constexpr int kHalf = 64;                                   // experts per phase-2 step: one 128-byte-wide R2 block
+    constexpr int kHalf = 64;                                   // experts per accumulator quarter: one 128-byte-wide block
+    constexpr int kSubs = FULL ? 4 : 1;                         // quarters per step
+    constexpr int kStep = kHalf * kSubs;                        // experts per step
+    constexpr int kFullStages = 3, kWBoxBytes = 64 * 128, kFullStageBytes = kXTileBytes + 4 * kWBoxBytes;
+    constexpr int kRing = FULL ? kFullRingBytes : kRingBytes;
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
     // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
     constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
@@ -136,21 +144,23 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kCandBytes = Sel::kCandBytes + (FILTER ? Sel::kZoneBytes : 0);
     constexpr int kMmas2 = FILTER ? kKSteps : 2 * kKSteps;      // exact modes: hi then lo into one accumulator
     // R2 blocks in flight: what the ring has room for next to the candidate buffers, at most 8 (unused by FULL)
-    constexpr int kStagesFit = (kRingBytes - kCandBytes) / kR2StageBytes;
+    constexpr int kStagesFit = (kRing - kCandBytes) / kR2StageBytes;
     constexpr int kStagesP2 = FULL ? 1 : (kStagesFit < 8 ? kStagesFit : 8);
     static_assert(FULL || kStagesP2 >= 2, "no room for the R2 pipeline");
-    constexpr int kCandOffset = FULL ? kStagesP1 * kP1StageBytes : 0;
-    static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRingBytes, "phase-2 layout does not fit");
+    constexpr int kCandOffset = FULL ? kFullStages * kFullStageBytes : 0;
+    static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRing, "phase-2 layout does not fit");
     // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
-    // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.
-    constexpr uint32_t kAccCols = 64, kZopCol0 = 128;
+    // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.  FULL: two 256-column
+    // accumulators, all 512 columns.
+    constexpr uint32_t kAccCols = FULL ? 256 : 64, kZopCol0 = 128;
+    constexpr uint32_t kTmemAlloc = FULL ? 512 : kTmemCols;
     constexpr float kLog2e = 1.4426950408889634f;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = (raw + 1023u) & ~1023u;            // 1024-aligned: the 128-B swizzle repeats every 1 KB
     uint8_t* ring_ptr = smem_raw + (ring - raw);
-    uint8_t* ctl = ring_ptr + kRingBytes;                    // control block
+    uint8_t* ctl = ring_ptr + kRing;                         // control block
     uint64_t* bars = reinterpret_cast<uint64_t*>(ctl);
     // barrier slots
     constexpr int kMaxStagesP1 = 4;
@@ -191,7 +201,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(kTmemCols)
+                     "r"(kTmemAlloc)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -202,24 +212,27 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     const uint32_t cand = ring + kCandOffset;                   // phase 2: candidate buffers
     const uint32_t r2ring = ring + kCandBytes;                  // phase 2: R2 stages
     // 64-expert steps of this CTA (the last one of the last tile is skipped when it lies wholly beyond M)
-    const int e_lo = tile_lo * kTileExperts;
-    const int e_hi = min(tile_hi * kTileExperts, p.M);
-    const int nsteps = (e_hi - e_lo + kHalf - 1) / kHalf;
+    constexpr int kTile = FULL ? kStep : kTileExperts;          // experts per tile of p.tiles_total
+    const int e_lo = tile_lo * kTile;
+    const int e_hi = min(tile_hi * kTile, p.M);
+    const int nsteps = (e_hi - e_lo + kStep - 1) / kStep;
 
     if (warp == 0) {
         // ===================================================================================== TMA producer
         if (lane == 0 && FULL) {
-            // standard router: for every 64-expert step, all k-tiles of X and of W[:, step]
+            // standard router: for every 256-expert step, all k-tiles of X and of W[:, step]
             bool ok = true;
             const int total = nsteps * ktiles1;
             for (int g = 0; g < total && ok; ++g) {
-                const int s = g % kStagesP1, it = g / ktiles1, kt = g % ktiles1;
-                if (g >= kStagesP1) ok = mbar_wait(bar(B_EMPTY1 + s), ((g / kStagesP1) - 1) & 1, abort_flag, p.status);
+                const int s = g % kFullStages, it = g / ktiles1, kt = g % ktiles1;
+                if (g >= kFullStages) ok = mbar_wait(bar(B_EMPTY1 + s), ((g / kFullStages) - 1) & 1, abort_flag, p.status);
                 if (!ok) break;
-                const uint32_t dst = ring + s * kP1StageBytes;
-                mbar_expect_tx(bar(B_FULL1 + s), kP1StageBytes);
+                const uint32_t dst = ring + s * kFullStageBytes;
+                mbar_expect_tx(bar(B_FULL1 + s), kFullStageBytes);
                 tma_load_2d(dst, &map_x, bar(B_FULL1 + s), kt * 64, tok0);            // 256 token rows x 64 columns
-                tma_load_2d(dst + kXTileBytes, &map_r2, bar(B_FULL1 + s), e_lo + it * kHalf, kt * 64);
+                for (int j = 0; j < 4; ++j)                                           // 64 k-rows x 4 x 64 experts
+                    tma_load_2d(dst + kXTileBytes + j * kWBoxBytes, &map_r2, bar(B_FULL1 + s), e_lo + it * kStep + j * kHalf,
+                                kt * 64);
             }
         } else if (lane == 0) {
             bool ok = true;
@@ -249,7 +262,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         constexpr uint32_t idesc1 = umma_idesc(64);
         constexpr uint32_t idesc2 = FILTER ? umma_idesc_f16(kHalf) : umma_idesc(kHalf);
         if constexpr (FULL) {
-            // standard router: per 64-expert step, K runs over all of h through the two k-tile stages
+            // standard router: per 256-expert step, K runs over all of h through the k-tile stages; each K = 16 slice
+            // is four N = 64 instructions, one per 64-expert box of the W tile and accumulator quarter
             const uint64_t xd = umma_desc_sw128(ring, 16, 1024), wd = umma_desc_sw128(ring + kXTileBytes, 8192, 1024);
             const uint32_t x_lo0 = (uint32_t)xd, x_hi = (uint32_t)(xd >> 32), w_lo0 = (uint32_t)wd, w_hi = (uint32_t)(wd >> 32);
             int g = 0;
@@ -261,18 +275,20 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
                 if (!ok) break;
                 for (int kt = 0; kt < ktiles1 && ok; ++kt, ++g) {
-                    const int s = g % kStagesP1;
-                    ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (g / kStagesP1) & 1, abort_flag, p.status));
+                    const int s = g % kFullStages;
+                    ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL1 + s), (g / kFullStages) & 1, abort_flag, p.status));
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t x_lo = x_lo0 + s * (kP1StageBytes >> 4), w_lo = w_lo0 + s * (kP1StageBytes >> 4);
+                    const uint32_t x_lo = x_lo0 + s * (kFullStageBytes >> 4), w_lo = w_lo0 + s * (kFullStageBytes >> 4);
 #pragma unroll
                     for (int a = 0; a < 2; ++a) {
                         if (a * 128 >= p.block_tokens) continue;
 #pragma unroll
                         for (int kk = 0; kk < 4; ++kk)
-                            tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
-                                                 w_lo + kk * (2048 >> 4), w_hi, idesc1, (kt | kk) != 0);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                tc_mma_bf16_ss_elect(tmem_base + a * kAccCols + j * kHalf, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
+                                                     w_lo + j * (kWBoxBytes >> 4) + kk * (2048 >> 4), w_hi, idesc1, (kt | kk) != 0);
                     }
                     tc_commit_elect(bar(B_EMPTY1 + s));
                 }
@@ -432,8 +448,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 
         const bool group_live = acc * 128 < p.block_tokens;
         for (int it = 0; it < nsteps && ok && group_live; ++it) {
-            const int e0 = e_lo + it * kHalf;
-            const bool ragged = e0 + kHalf > p.M;
+            int e0 = e_lo + it * kStep;
+            bool ragged = e0 + kHalf > p.M;
             float va[16], vb[16];
             // ---- one 16-column chunk: group-of-four maxima, optional online softmax update, candidate scan
             auto process = [&](float (&v)[16], int col0) {
@@ -490,23 +506,30 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 continue;
             }
             tc_fence_after();
-            // columns 0-31: the load of the next 16 columns is in flight while the current 16 are processed
-            tmem_ld16(t_lane, va);
-            tmem_ld_wait16(va);
-            tmem_ld16(t_lane + 16, vb);
-            process(va, e0);
-            tmem_ld_wait16(vb);
-            tmem_ld16(t_lane + 32, va);
-            process(vb, e0 + 16);
-            // columns 32-63: both halves are brought into registers first; the accumulator can then be handed back,
-            // and the next step's MMAs run while these 32 columns are processed
-            tmem_ld_wait16(va);
-            tmem_ld16(t_lane + 48, vb);
-            tmem_ld_wait16(vb);
-            tc_fence_before();
-            mbar_arrive(bar(B_ACCE + acc));
-            process(va, e0 + 32);
-            process(vb, e0 + 48);
+#pragma unroll 1
+            for (int sub = 0; sub < kSubs; ++sub, e0 += kHalf) {      // (one 64-column quarter unless FULL)
+                const uint32_t t_sub = t_lane + sub * kHalf;
+                ragged = e0 + kHalf > p.M;
+                // columns 0-31: the load of the next 16 columns is in flight while the current 16 are processed
+                tmem_ld16(t_sub, va);
+                tmem_ld_wait16(va);
+                tmem_ld16(t_sub + 16, vb);
+                process(va, e0);
+                tmem_ld_wait16(vb);
+                tmem_ld16(t_sub + 32, va);
+                process(vb, e0 + 16);
+                // columns 32-63: both halves are brought into registers first; after the last quarter the accumulator
+                // can then be handed back, and the next step's MMAs run while these 32 columns are processed
+                tmem_ld_wait16(va);
+                tmem_ld16(t_sub + 48, vb);
+                tmem_ld_wait16(vb);
+                if (sub == kSubs - 1) {
+                    tc_fence_before();
+                    mbar_arrive(bar(B_ACCE + acc));
+                }
+                process(va, e0 + 32);
+                process(vb, e0 + 48);
+            }
             STAT(st_tproc += clock64() - tw1;)
         }
         S.fold();
@@ -758,7 +781,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemAlloc) : "memory");
     }
 }
 
@@ -826,11 +849,12 @@ int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& 
                cudaStream_t st, bool clear_counts)
 {
     static unsigned long long configured = 0;   // one bit per device, per instantiation; guarded by the API mutex
+    constexpr int smem_bytes = (FULL ? kFullRingBytes : kRingBytes) + 2048;    // + alignment slack + control block
     auto kern = route_tcgen05_kernel<RPAD, KCAP, LSE, FULL, FILTER>;
     int dev = 0;
     cudaGetDevice(&dev);
     if (!(configured >> (dev & 63) & 1ull)) {
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes) != cudaSuccess)
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes) != cudaSuccess)
             return MORE_ERR_CUDA;
         configured |= 1ull << (dev & 63);
     }
@@ -838,7 +862,7 @@ int launch_one(const CUtensorMap& mx, const CUtensorMap& m1, const CUtensorMap& 
     if (clear_counts &&
         cudaMemsetAsync(kp.out_counts, 0, (size_t)kp.M * sizeof(int32_t), st) != cudaSuccess)
         return MORE_ERR_CUDA;
-    kern<<<ctas, kThreads, kSmemBytes, st>>>(mx, m1, m2, kp);
+    kern<<<ctas, kThreads, smem_bytes, st>>>(mx, m1, m2, kp);
     count_launch(1);
     return cudaGetLastError() == cudaSuccess ? MORE_OK : MORE_ERR_CUDA;
 }
@@ -927,7 +951,7 @@ int launch_paired(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scrat
     kp.T = a.T; kp.h = a.h; kp.r = a.r; kp.M = a.M; kp.k = a.k; kp.gate_mode = a.gate_mode; kp.msplit = p.msplit;
     kp.block_tokens = p.block_tokens;
     kp.x_rows = x_rows;
-    kp.tiles_total = (a.M + kTileExperts - 1) / kTileExperts;
+    kp.tiles_total = a.full ? (a.M + 255) / 256 : (a.M + kTileExperts - 1) / kTileExperts;
     kp.out_idx = a.out_idx; kp.out_gate = a.out_gate; kp.out_counts = a.out_counts;
     kp.out_topval = a.out_topval; kp.out_lse = a.out_lse;
     kp.status = ctx.status;
