@@ -336,10 +336,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
                 if (!ok) break;
                 tc_fence_after();
-#pragma unroll
-                for (int j = 0; j < kMmas2; ++j)            // K runs over [hi | lo]: 8 columns of A, 16 rows of B per step
-                    tc_mma_bf16_ts_elect(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64 + j * 8,
-                                         b_lo + (j % kKSteps) * (2048 >> 4), b_hi, idesc2, j != 0);
+                // K runs over [hi | lo]: 8 columns of A, 16 rows of B per instruction; one instruction sequence, one election
+                tc_mma_buffer_ts<kMmas2, kKSteps>(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64, b_lo, b_hi, idesc2);
                 tc_commit_elect(bar(B_ACCF + a));
             }
             if (!ok) break;
