@@ -234,7 +234,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
 #else
     const bool filter_ok = false;
 #endif
-    const double c_lat = want_lse ? 260.0 : 190.0, c_iss = want_lse ? 120.0 : 62.0;
+    const double c_lat = want_lse ? 260.0 : 190.0, c_iss = want_lse ? 76.0 : 56.0;
     double best = 1e300;
     Plan bp = *p;
     for (int bt = 512; bt >= 32; bt -= 32) {
