@@ -35,12 +35,14 @@ def _run(case, msplit=0, gate_mode=None):
 
 @pytest.mark.parametrize("gate_mode", [0, 1])
 @pytest.mark.parametrize("T,h,M,k", [
-    (256, 128, 256, 2),        # one CTA, two k-tiles
+    (256, 128, 256, 2),        # one CTA, one full 256-expert step, two k-tiles
     (300, 136, 200, 4),        # ragged everywhere: h not a multiple of 64, M not of 64, T not of 32
-    (1000, 512, 1024, 8),      # several CTAs, eight k-tiles through two stages
+    (1000, 512, 1024, 8),      # several CTAs, eight k-tiles through three stages
     (2500, 64, 4096, 8),       # one k-tile per step
     (129, 256, 72, 16),        # list capacity 16, a token group with one live row
     (64, 384, 64, 32),         # list capacity 32, a single step
+    (600, 192, 1000, 8),       # four 256-expert steps, the last one ragged (232 experts)
+    (260, 128, 520, 4),        # three steps, eight live columns in the last; a second token group with four rows
 ])
 def test_full_router_matches_oracle(T, h, M, k, gate_mode):
     case = inputs.full_rank_case(T, h, M, k, gate_mode, seed=5)
