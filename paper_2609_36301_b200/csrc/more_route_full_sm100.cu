@@ -50,6 +50,11 @@ namespace {
 #ifndef MORE_CAND_CAP
 #define MORE_CAND_CAP 8
 #endif
+// 1: the low-rank router keeps z (the A operand of phase 2) in shared memory, which frees tensor memory for a second
+// accumulator per token group; 0: z in tensor memory, one accumulator per group
+#ifndef MORE_PAIRED_DBL
+#define MORE_PAIRED_DBL 1
+#endif
 // fused standard router: three stages of (256 x 64 X tile + 64 x 256 W tile) and six candidate slots per token
 constexpr int kFullRingBytes = 3 * (kXTileBytes + 4 * 64 * 128) + 6 * kEpilogueThreads * 20;
 constexpr int kFallbackSlots = 8;      // tokens re-routed per round of the filter's fallback (one per epilogue warp)
@@ -136,6 +141,15 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kRing = FULL ? kFullRingBytes : kRingBytes;
     constexpr int kR2StageBytes = RPAD * 128;                   // RPAD rows x 64 experts
     // candidate slots per token (the standard router keeps the two 40 KB k-tile stages next to the buffers)
+    // DBL (r <= 32): z is written to shared memory as one K-major 128 x 64 bf16 tile per token group (a row is
+    // [hi | lo] of one token, the layout of an X tile) and read by the phase-2 MMAs from there, so each group has two
+    // 64-column accumulators: the MMAs of step n + 1 run while the group still selects from step n, and a warp that
+    // stops to fold its candidates no longer stalls the group's next accumulator.  (At r = 64 the tiles take 64 KB,
+    // which leaves room for six candidate slots and two R2 stages only: measured slower, 390 against 375 us on c3.
+    // With the softmax sweep the epilogue is bound by its instructions, not by the hand-over: no gain, so not used.)
+    constexpr bool DBL = !FULL && !FILTER && !LSE && RPAD <= 32 && (MORE_PAIRED_DBL != 0);
+    constexpr int kZopTileBytes = 128 * 128;                    // 128 tokens x 64 bf16
+    constexpr int kZopBytes = DBL ? 2 * kZopTileBytes : 0;      // [group]
     constexpr int kCandCap = FULL ? 6 : MORE_CAND_CAP;
     using Sel = Selector<KCAP, FILTER, kEpilogueThreads, kCandCap, 4>;
     STAT(constexpr int kCandValStride = Sel::kCandValStride;)
@@ -144,15 +158,17 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kCandBytes = Sel::kCandBytes + (FILTER ? Sel::kZoneBytes : 0);
     constexpr int kMmas2 = FILTER ? kKSteps : 2 * kKSteps;      // exact modes: hi then lo into one accumulator
     // R2 blocks in flight: what the ring has room for next to the candidate buffers, at most 8 (unused by FULL)
-    constexpr int kStagesFit = (kRing - kCandBytes) / kR2StageBytes;
+    constexpr int kStagesFit = (kRing - kZopBytes - kCandBytes) / kR2StageBytes;
     constexpr int kStagesP2 = FULL ? 1 : (kStagesFit < 8 ? kStagesFit : 8);
     static_assert(FULL || kStagesP2 >= 2, "no room for the R2 pipeline");
-    constexpr int kCandOffset = FULL ? kFullStages * kFullStageBytes : 0;
+    constexpr int kCandOffset = FULL ? kFullStages * kFullStageBytes : kZopBytes;
     static_assert(kCandOffset + kCandBytes + (FULL ? 0 : kStagesP2 * kR2StageBytes) <= kRing, "phase-2 layout does not fit");
     // Tensor-memory columns of this CTA: [0, 128) the two 64-column fp32 accumulators (phase 1: z, phase 2: logits),
     // [128, 256) the two A operands of phase 2, z as bf16 [hi | lo], two K-elements per column.  FULL: two 256-column
     // accumulators, all 512 columns.
     constexpr uint32_t kAccCols = FULL ? 256 : 64, kZopCol0 = 128;
+    constexpr uint32_t kAccStride = DBL ? 128 : kAccCols;       // columns between the two groups' accumulators
+    constexpr int kAccBufs = DBL ? 2 : 1;                       // accumulators per group (64 columns apart)
     constexpr uint32_t kTmemAlloc = FULL ? 512 : kTmemCols;
     constexpr float kLog2e = 1.4426950408889634f;
 
@@ -165,8 +181,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // barrier slots
     constexpr int kMaxStagesP1 = 4;
     constexpr int B_FULL1 = 0, B_EMPTY1 = B_FULL1 + kMaxStagesP1, B_ZACC = B_EMPTY1 + kMaxStagesP1, B_ZOP = B_ZACC + 1,
-                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 2,
-                  B_COUNT = B_ACCE + 2;
+                  B_FULL2 = B_ZOP + 1, B_EMPTY2 = B_FULL2 + 8, B_ACCF = B_EMPTY2 + 8, B_ACCE = B_ACCF + 4,
+                  B_COUNT = B_ACCE + 4;                  // accumulator barriers: [group * kAccBufs + buffer]
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(ctl + B_COUNT * 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(ctl + B_COUNT * 8 + 4);
     int* last_flag = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 8);
@@ -193,7 +209,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         mbar_init(bar(B_ZACC), 1);
         mbar_init(bar(B_ZOP), kEpilogueThreads);
         for (int i = 0; i < 8; ++i) { mbar_init(bar(B_FULL2 + i), 1); mbar_init(bar(B_EMPTY2 + i), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads / 2); }
+        for (int i = 0; i < 4; ++i) { mbar_init(bar(B_ACCF + i), 1); mbar_init(bar(B_ACCE + i), kEpilogueThreads / 2); }
         *abort_flag = 0;
         *last_flag = 0;
         *flagged = 0;
@@ -210,7 +226,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     const uint32_t cand = ring + kCandOffset;                   // phase 2: candidate buffers
-    const uint32_t r2ring = ring + kCandBytes;                  // phase 2: R2 stages
+    const uint32_t r2ring = ring + (FULL ? 0 : kCandOffset) + kCandBytes;     // phase 2: R2 stages
     // 64-expert steps of this CTA (the last one of the last tile is skipped when it lies wholly beyond M)
     constexpr int kTile = FULL ? kStep : kTileExperts;          // experts per tile of p.tiles_total
     const int e_lo = tile_lo * kTile;
@@ -313,7 +329,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     if (a * 128 >= p.x_rows) continue;      // a 128-row X tile has no second token group
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk)      // A: +32 B per K = 16; B: 16 K-rows of 128 B
-                        tc_mma_bf16_ss_elect(tmem_base + a * kAccCols, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
+                        tc_mma_bf16_ss_elect(tmem_base + a * kAccStride, x_lo + a * (16384 >> 4) + kk * 2, x_hi,
                                              r_lo + kk * (2048 >> 4), r_hi, idesc1, (kt | kk) != 0);
                 }
                 tc_commit_elect(bar(B_EMPTY1 + s));
@@ -324,6 +340,8 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         tc_fence_after();
         const uint64_t bd0 = umma_desc_sw128(r2ring, 8192, 1024);
         const uint32_t b_lo0 = (uint32_t)bd0, b_hi = (uint32_t)(bd0 >> 32);
+        const uint64_t zd0 = umma_desc_sw128(ring, 16, 1024);             // DBL: the z tiles, K-major like an X tile
+        const uint32_t z_lo0 = (uint32_t)zd0, z_hi = (uint32_t)(zd0 >> 32);
         for (int it = 0; it < nsteps && ok; ++it) {
             const int s = it % kStagesP2;
             ok = __all_sync(kFullMask, mbar_wait(bar(B_FULL2 + s), (it / kStagesP2) & 1, abort_flag, p.status));
@@ -332,13 +350,26 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
             for (int a = 0; a < 2; ++a) {
                 if (a * 128 >= p.block_tokens) continue;     // a group without tokens takes no part in phase 2
-                // accumulator a is free once its 128 epilogue threads have read the previous step out of it
-                ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
-                if (!ok) break;
-                tc_fence_after();
-                // K runs over [hi | lo]: 8 columns of A, 16 rows of B per instruction; one instruction sequence, one election
-                tc_mma_buffer_ts<kMmas2, kKSteps>(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64, b_lo, b_hi, idesc2);
-                tc_commit_elect(bar(B_ACCF + a));
+                if constexpr (DBL) {
+                    // accumulator (a, it & 1) is free once its 128 epilogue threads have read step it - 2 out of it
+                    const int buf = it & 1;
+                    ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a * 2 + buf), ((it >> 1) & 1) ^ 1, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    // A from shared memory: K runs over the row [hi | lo], +32 B per K = 16
+                    if constexpr (RPAD <= 32)
+                        tc_mma_buffer_ss<kMmas2, kKSteps>(tmem_base + a * kAccStride + buf * kAccCols,
+                                                          z_lo0 + a * (kZopTileBytes >> 4), z_hi, b_lo, b_hi, idesc2);
+                    tc_commit_elect(bar(B_ACCF + a * 2 + buf));
+                } else {
+                    // accumulator a is free once its 128 epilogue threads have read the previous step out of it
+                    ok = __all_sync(kFullMask, ok && mbar_wait(bar(B_ACCE + a), (it & 1) ^ 1, abort_flag, p.status));
+                    if (!ok) break;
+                    tc_fence_after();
+                    // K runs over [hi | lo]: 8 columns of A, 16 rows of B per instruction; one instruction sequence, one election
+                    tc_mma_buffer_ts<kMmas2, kKSteps>(tmem_base + a * kAccCols, tmem_base + kZopCol0 + a * 64, b_lo, b_hi, idesc2);
+                    tc_commit_elect(bar(B_ACCF + a));
+                }
             }
             if (!ok) break;
             tc_commit_elect(bar(B_EMPTY2 + s));
@@ -353,7 +384,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         const int64_t row = (int64_t)tok0 + row_in_blk;
         const bool row_live = row_in_blk < p.block_tokens && row < p.T;     // rows past the block belong to the next CTA
         const bool warp_live = acc * 128 + q * 32 < p.block_tokens;         // warp-uniform: block_tokens is a multiple of 32
-        const uint32_t t_lane = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccCols;
+        const uint32_t t_lane0 = tmem_base + ((uint32_t)(q * 32) << 16) + acc * kAccStride;    // the group's (first) accumulator
         const uint32_t t_zop = tmem_base + ((uint32_t)(q * 32) << 16) + kZopCol0 + acc * 64;
         STAT(const long long st_k0 = clock64();)
         bool ok = FULL ? true : mbar_wait(bar(B_ZACC), 0, abort_flag, p.status);
@@ -373,7 +404,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
                 for (int c = 0; c < RPAD / 16; ++c) {
                     float z[16];
-                    tmem_ld16(t_lane + c * 16, z);
+                    tmem_ld16(t_lane0 + c * 16, z);
                     tmem_ld_wait16(z);
 #pragma unroll
                     for (int e = 0; e < 16; ++e) zmax = fmaxf(zmax, fabsf(z[e]));
@@ -386,7 +417,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
 #pragma unroll
             for (int c = 0; c < RPAD / 16; ++c) {
                 float z[16];
-                tmem_ld16(t_lane + c * 16, z);
+                tmem_ld16(t_lane0 + c * 16, z);
                 tmem_ld_wait16(z);
                 uint32_t hi[8], lo[8];
 #pragma unroll
@@ -412,16 +443,35 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                         lo[e] = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
                     }
                 }
-                tmem_st8(t_zop + c * 8, hi);
-                if (FILTER) {
-                    zlo[(2 * c) * kEpilogueThreads] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-                    zlo[(2 * c + 1) * kEpilogueThreads] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                if constexpr (DBL) {
+                    // row `row_in_acc` of the group's tile (128-byte rows, 1 KB per 8 rows): ranks 16c .. 16c+15 of hi are
+                    // the 16-byte chunks 2c and 2c+1, those of lo follow the RPAD/8 chunks of hi; a chunk is stored at
+                    // chunk index ^ (row % 8): the 128-byte swizzle
+                    const uint32_t zrow = ring + acc * kZopTileBytes + (row_in_acc >> 3) * 1024 + (row_in_acc & 7) * 128;
+                    const uint32_t x7 = row_in_acc & 7;
+                    const uint32_t h0 = ((2 * c) ^ x7) * 16, h1 = ((2 * c + 1) ^ x7) * 16;
+                    const uint32_t l0 = ((RPAD / 8 + 2 * c) ^ x7) * 16, l1 = ((RPAD / 8 + 2 * c + 1) ^ x7) * 16;
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zrow + h0), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zrow + h1), "r"(hi[4]), "r"(hi[5]), "r"(hi[6]), "r"(hi[7]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zrow + l0), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(zrow + l1), "r"(lo[4]), "r"(lo[5]), "r"(lo[6]), "r"(lo[7]) : "memory");
                 } else {
-                    tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                    tmem_st8(t_zop + c * 8, hi);
+                    if (FILTER) {
+                        zlo[(2 * c) * kEpilogueThreads] = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+                        zlo[(2 * c + 1) * kEpilogueThreads] = make_uint4(lo[4], lo[5], lo[6], lo[7]);
+                    } else {
+                        tmem_st8(t_zop + RPAD / 2 + c * 8, lo);
+                    }
                 }
             }
-            tmem_st_wait();
-            tc_fence_before();
+            if constexpr (DBL) {
+                fence_async_smem();              // the tiles are read by the tensor core (async proxy)
+                tc_fence_before();               // ... and this thread's loads of z are complete
+            } else {
+                tmem_st_wait();
+                tc_fence_before();
+            }
             mbar_arrive(bar(B_ZOP));
             if (FILTER) {
                 // |approximate - fp32 logit| (both in the scaled units of this token) <= |z - hi|_2 |R2_j|_2 for the
@@ -496,11 +546,15 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 }
             };
             STAT(const long long tw0 = clock64();)
-            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + acc), it & 1, abort_flag, p.status));
+            // the accumulator of this step: the group's only one, or (DBL) its buffer it & 1, in use every other step
+            const int abuf = DBL ? (it & 1) : 0;
+            const int abar = acc * kAccBufs + abuf;
+            const uint32_t t_lane = t_lane0 + abuf * kAccCols;
+            ok = __all_sync(kFullMask, mbar_wait(bar(B_ACCF + abar), (DBL ? (it >> 1) : it) & 1, abort_flag, p.status));
             STAT(const long long tw1 = clock64(); st_twait += tw1 - tw0;)
             if (!ok) break;
             if (!warp_live) {                                // nothing to select for these rows: just hand the buffer back
-                mbar_arrive(bar(B_ACCE + acc));
+                mbar_arrive(bar(B_ACCE + abar));
                 continue;
             }
             tc_fence_after();
@@ -523,7 +577,7 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 tmem_ld_wait16(vb);
                 if (sub == kSubs - 1) {
                     tc_fence_before();
-                    mbar_arrive(bar(B_ACCE + acc));
+                    mbar_arrive(bar(B_ACCE + abar));
                 }
                 process(va, e0 + 32);
                 process(vb, e0 + 48);

@@ -319,6 +319,30 @@ __device__ __forceinline__ void tc_mma_buffer_ts(uint32_t d, uint32_t a0, uint32
 #undef MORE_MMA_STEP
 #undef MORE_MMA_OPEN
 
+// The same with the A operand in shared memory (K-major, 32 bytes per K = 16 step): a_lo / a_hi are the two words of
+// the A descriptor of the first step.  NM = 2 K-steps wrapping after 1, or 4 wrapping after 2.
+#define MORE_MMA_STEP_SS(AOFF, BOFF, PRED)                                                           \
+    "add.u32 al, %1, " #AOFF ";\n\tmov.b64 ad, {al, %2};\n\tadd.u32 bl, %3, " #BOFF ";\n\tmov.b64 bd, {bl, %4};\n\t" \
+    "@pe tcgen05.mma.cta_group::1.kind::f16 [%0], ad, bd, %5, " #PRED ";\n\t"
+#define MORE_MMA_OPEN_SS                                                                             \
+    "{\n\t.reg .pred pe, pt, pf;\n\t.reg .b64 ad, bd;\n\t.reg .b32 al, bl;\n\t"                  \
+    "setp.eq.u32 pt, 0, 0;\n\tsetp.ne.u32 pf, 0, 0;\n\telect.sync _|pe, 0xffffffff;\n\t"
+template <int NM, int KS>
+__device__ __forceinline__ void tc_mma_buffer_ss(uint32_t d, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                 uint32_t idesc)
+{
+    static_assert((NM == 2 && KS == 1) || (NM == 4 && KS == 2), "unsupported MMA sequence");
+    if constexpr (NM == 2)
+        asm volatile(MORE_MMA_OPEN_SS MORE_MMA_STEP_SS(0, 0, pf) MORE_MMA_STEP_SS(2, 0, pt) "}"
+                     ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+    else
+        asm volatile(MORE_MMA_OPEN_SS MORE_MMA_STEP_SS(0, 0, pf) MORE_MMA_STEP_SS(2, 128, pt) MORE_MMA_STEP_SS(4, 0, pt)
+                     MORE_MMA_STEP_SS(6, 128, pt) "}"
+                     ::"r"(d), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc) : "memory");
+}
+#undef MORE_MMA_STEP_SS
+#undef MORE_MMA_OPEN_SS
+
 }  // namespace
 
 // 2-D bf16 row-major tensor [rows][cols] -> TMA descriptor with box = box_cols x box_rows, 128-byte swizzle, zero
