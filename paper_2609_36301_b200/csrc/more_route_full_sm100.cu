@@ -145,7 +145,9 @@ route_tcgen05_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     // [hi | lo] of one token, the layout of an X tile) and read by the phase-2 MMAs from there, so each group has two
     // 64-column accumulators: the MMAs of step n + 1 run while the group still selects from step n, and a warp that
     // stops to fold its candidates no longer stalls the group's next accumulator.  (At r = 64 the tiles take 64 KB,
-    // which leaves room for six candidate slots and two R2 stages only: measured slower, 390 against 375 us on c3;
+    // which leaves room for six candidate slots and two R2 stages only: measured slower, 390 against 375 us on c3, and
+    // 380 with the overflow check run twice per chunk so that six slots fold as rarely as eight: the waits then move
+    // from the accumulators to the two R2 stages;
     // so is keeping only the hi half in shared memory, lo in 32 tensor-memory columns and sweeping 48 experts per step
     // with two 48-column accumulators: 387 us, a third more steps with their hand-overs.
     // With the softmax sweep the epilogue is bound by its instructions, not by the hand-over: no gain, so not used.)
