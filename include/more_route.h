@@ -158,9 +158,9 @@ int more_route_psum(const void* X, const void* R1, const void* R2, int T, int h,
 /*
  * more_route_full -- the fused STANDARD (full-rank) router, g(x) = softmax(TopK(R x)): the same sweep without the
  * low-rank bottleneck (Algorithm 1 with the contraction running over K = h instead of r; the paper's "fused standard
- * MoE" comparison).  Logits l = X W with W = R^T stored [h][M] row-major; they are produced 64 experts at a time by
+ * MoE" comparison).  Logits l = X W with W = R^T stored [h][M] row-major; they are produced 256 experts at a time by
  * accumulating over all of h on the tensor cores, and selected, gated and counted exactly as in more_route.  The
- * T x M logits never reach memory, but X is re-read (from L2) once per 64-expert step, so unlike the low-rank router
+ * T x M logits never reach memory, but X is re-read (from L2) once per 256-expert step, so unlike the low-rank router
  * this one does a full T x h x M contraction.
  *
  *   X           device bf16 [T][h];  W  device bf16 [h][M];  both 16-byte aligned; h and M multiples of 8, k <= 32
