@@ -548,6 +548,7 @@ def main():
                                                     bound=r["bound"], roofline_frac=r["frac"], msplit=oplan.msplit,
                                                     ctas=oplan.ctas, block_tokens=oplan.block_tokens,
                                                     expert_ranges=oplan.expert_ranges,
+                                                    kernel="route_tcgen05_kernel" if oplan.paired else "route_lowrank_kernel",
                                                     host_us_per_call=host_us_per_call(mr, torch, obufs, ocase.k, gm, stream, 100),
                                                     **diagnostic_bounds(ocase.T, ocase.M, gm, ocnt.get("warp_instr_per_chunk"),
                                                                         clocks.get("sm_mhz")))
