@@ -122,8 +122,40 @@ int route_device_locked(const RouteArgs& a, int path, int msplit)
     if (rc != MORE_OK) return rc;
     Plan plan;
     const bool want_lse = a.gate_mode == MORE_GATE_FULL_SOFTMAX || a.out_lse != nullptr;
-    rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, want_lse, a.full, path, msplit, ctx->sm_count, &plan);
-    if (rc != MORE_OK) return rc;
+    {
+        // The planner walks a few thousand candidates for a decode-sized shape (tens of microseconds, comparable with
+        // the kernel it plans); repeated calls with the same shape take the plan from a small cache.  Guarded by the
+        // API mutex like everything here.
+        struct PlanKey {
+            int T, h, r, M, k, gate_mode, want_lse, full, path, msplit, sm_count;
+            bool operator==(const PlanKey& o) const
+            {
+                return T == o.T && h == o.h && r == o.r && M == o.M && k == o.k && gate_mode == o.gate_mode &&
+                       want_lse == o.want_lse && full == o.full && path == o.path && msplit == o.msplit && sm_count == o.sm_count;
+            }
+        };
+        constexpr int kPlanCache = 16;
+        static PlanKey keys[kPlanCache];
+        static Plan plans[kPlanCache];
+        static int used = 0, next = 0;
+        const PlanKey key{a.T, a.h, a.r, a.M, a.k, a.gate_mode, want_lse ? 1 : 0, a.full ? 1 : 0, path, msplit, ctx->sm_count};
+        int hit = -1;
+        for (int i = 0; i < used; ++i)
+            if (keys[i] == key) { hit = i; break; }
+#ifdef MORE_DEV
+        hit = -1;                                  // development builds re-plan every call (MORE_PLAN / MORE_KERNEL overrides)
+#endif
+        if (hit >= 0) {
+            plan = plans[hit];
+        } else {
+            rc = make_plan(a.T, a.h, a.r, a.M, a.k, a.gate_mode, want_lse, a.full, path, msplit, ctx->sm_count, &plan);
+            if (rc != MORE_OK) return rc;
+            keys[next] = key;
+            plans[next] = plan;
+            next = (next + 1) % kPlanCache;
+            if (used < kPlanCache) ++used;
+        }
+    }
     const size_t need = plan.path != MORE_PATH_TCGEN05
                             ? generic_scratch_bytes(a)
                             : (a.full ? full_scratch_bytes(a, plan)
