@@ -39,10 +39,11 @@ def test_small_token_counts(T, h, r, M, k, gate_mode):
     _route_and_check(case, 0)
 
 
-@pytest.mark.parametrize("T", [1, 40, 64, 72])
+@pytest.mark.parametrize("T", [1, 40, 64, 72, 100, 128, 250])
 @pytest.mark.parametrize("msplit", [2, 8, 16])
 def test_small_token_counts_with_forced_split(T, msplit):
-    """Forced CTA splits of a 4096-expert sweep: 2 (serial merge), 8 and 16 (fanned-out network merge)."""
+    """Forced CTA splits of a 4096-expert sweep: 2 (serial merge), 8 and 16 (fanned-out network merge, 2 to 16 threads
+    per token depending on the block size the plan picks)."""
     case = inputs.gaussian_case(T, 512, 32, 4096, 8, 1, seed=2000 + T + msplit)
     plan = mr.more_route_plan_ex(T, 512, 32, 4096, 8, 1, True, mr.PATH_TCGEN05, msplit)
     assert plan.msplit == msplit
@@ -61,3 +62,14 @@ def test_equal_logits_across_expert_ranges_keep_the_lower_id():
     for msplit in (0, 4, 16):
         st = _route_and_check(case, msplit)
         assert not st["differs_mask"].any()
+
+
+@pytest.mark.parametrize("T,h,r,M,k", [(1024, 1024, 32, 8192, 8), (512, 512, 32, 65536, 8), (1000, 256, 16, 16384, 4)])
+@pytest.mark.parametrize("gate_mode", [0, 1])
+def test_mid_sized_batches_split_over_many_ctas(T, h, r, M, k, gate_mode):
+    """A few hundred to a thousand tokens with many experts: the plan splits every token block over 8 or more CTAs with
+    64 to 128 tokens per block, so the last-arriver merge runs with two to four threads per token."""
+    case = inputs.gaussian_case(T, h, r, M, k, gate_mode, seed=3000 + T)
+    plan = mr.more_route_plan_ex(T, h, r, M, k, gate_mode, True, mr.PATH_TCGEN05, 0)
+    assert not plan.paired and plan.msplit >= 8
+    _route_and_check(case, 0)
