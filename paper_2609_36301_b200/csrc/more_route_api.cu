@@ -341,11 +341,11 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
     } else {
         // Two kernels serve the low-rank router (measured on B200, both gate modes, T from 8 k to 64 k tokens): the
         // grouped kernel (one CTA per SM, up to four token groups / expert ranges side by side) wins while an SM has
-        // fewer than ~160 tokens, and up to ~320 tokens per SM when no softmax sweep is wanted and the expert count is
-        // moderate; the paired kernel (256-token CTAs, two per SM, 64-expert steps) wins on everything larger.
+        // fewer than ~160 tokens, and up to ~320 tokens per SM when the expert count is moderate (M <= 32768); the paired
+        // kernel (256-token CTAs, two per SM, 64-expert steps) wins on everything larger.
         p.block_tokens = 0;
         const long long per_sm = ((long long)T + sm_count - 1) / sm_count;
-        bool grouped = per_sm < 160 || (!want_lse && per_sm < 320 && M <= 32768);
+        bool grouped = per_sm < 160 || (per_sm < 320 && M <= 32768);
 #ifdef MORE_DEV
         if (const char* kk = getenv("MORE_KERNEL")) grouped = kk[0] == 'g';
 #endif
