@@ -339,13 +339,22 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
     if (full) {
         plan_dense(T, h, M, msplit, sm_count, &p);
     } else {
-        // Two kernels serve the low-rank router (measured on B200, both gate modes, T from 8 k to 64 k tokens): the
-        // grouped kernel (one CTA per SM, up to four token groups / expert ranges side by side) wins while an SM has
-        // fewer than ~160 tokens, and up to ~320 tokens per SM when the expert count is moderate (M <= 32768); the paired
-        // kernel (256-token CTAs, two per SM, 64-expert steps) wins on everything larger.
+        // Two kernels serve the low-rank router.  Measured on B200 over T = 2 k ... 64 k tokens, M = 1 k ... 64 k
+        // experts, r = 16, 32, 64 and both gates: the grouped kernel (one CTA per SM, up to four token groups / expert
+        // ranges side by side) wins while an SM has fewer than ~120 tokens; between that and ~260 tokens per SM it
+        // wins for up to ~8 k experts, and with the softmax sweep (whose epilogue is bound by its own instructions
+        // rather than by the accumulator hand-over) up to ~250 tokens per SM for any expert count when its 128-token
+        // groups fill evenly; the paired kernel
+        // (256-token CTAs, two per SM, 64-expert steps, two accumulators per group at r <= 32) wins on the rest.
         p.block_tokens = 0;
         const long long per_sm = ((long long)T + sm_count - 1) / sm_count;
-        bool grouped = per_sm < 160 || (per_sm < 320 && M <= 32768);
+        // (a CTA of the grouped kernel holds its tokens in groups of 128: with, say, 167 tokens per SM the second
+        // group of every CTA is two thirds empty, and the kernel loses what it otherwise gains)
+        const bool even_fill = per_sm % 128 == 0 || per_sm % 128 >= 80;
+        bool grouped;
+        if (per_sm < 120) grouped = true;
+        else if (M <= 8192) grouped = per_sm < (want_lse ? 320 : 260);
+        else grouped = want_lse && per_sm < 250 && even_fill;
 #ifdef MORE_DEV
         if (const char* kk = getenv("MORE_KERNEL")) grouped = kk[0] == 'g';
 #endif
