@@ -354,7 +354,7 @@ int make_plan(int T, int h, int r, int M, int k, int gate_mode, bool want_lse, b
         bool grouped;
         if (per_sm < 120) grouped = true;
         else if (M <= 8192) grouped = per_sm < (want_lse ? 320 : 260);
-        else grouped = want_lse && per_sm < 250 && even_fill;
+        else grouped = (want_lse || M <= 16384) && per_sm < 250 && even_fill;      // (M = 16 k with the top-k gate: a tie)
 #ifdef MORE_DEV
         if (const char* kk = getenv("MORE_KERNEL")) grouped = kk[0] == 'g';
 #endif
