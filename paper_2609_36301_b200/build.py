@@ -24,8 +24,11 @@ def build(force: bool = False, verbose: bool = False, out: str | None = None, de
     """Compile the CUDA sources if the library is missing or older than any source; return its path.
 
     ``defines`` adds ``-D`` switches (the diagnostic builds: ``MORE_STATS`` for event and clock counters,
-    ``MORE_EXP_NOSCAN`` / ``MORE_EXP_NOPROC`` for the epilogue with its candidate handling, or everything but the
-    tensor-memory loads, compiled out); such a build goes to ``out``, never over the product library."""
+    ``MORE_EXP_NOSCAN`` / ``MORE_EXP_NOPROC`` / ``MORE_EXP_NOFOLD`` for the epilogue with its candidate handling,
+    everything but the tensor-memory loads, or its folds compiled out; ``MORE_DEV`` for the ``MORE_KERNEL=p|g`` and
+    ``MORE_PLAN=block_tokens,es,msplit,filter`` environment overrides of the launch plan; ``MORE_PAIRED_DBL=0`` for the
+    paired kernel with z in tensor memory at every rank; ``MORE_WITH_FILTER`` for the experimental filter sweep;
+    ``MORE_CAND_CAP=n`` candidate slots per token); such a build goes to ``out``, never over the product library."""
     target = out or LIB_PATH
     if defines and target == LIB_PATH:
         raise ValueError("a diagnostic build needs its own output path")
