@@ -70,7 +70,7 @@ constexpr int kEpiThreads = 128 * kGroups;
 constexpr int kFirstEpiWarp = 2;
 constexpr int kRThreads = 32 * kFirstEpiWarp + kEpiThreads;   // TMA warp, phase-1 MMA warp, 16 epilogue warps
 constexpr int kRRing = 208 * 1024;                 // shared-memory working area
-constexpr int kRSmem = kRRing + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/;
+constexpr int kRSmem = kRRing + 1024 /*alignment slack*/ + 1024 /*barriers, flags*/ + 4096 /*published thresholds*/;
 constexpr int kGroupCols = 128;                    // tensor-memory columns per group
 constexpr int kBufCols = 32;                       // one accumulator buffer of the ring
 #ifndef MORE_CAND_CAP
@@ -342,7 +342,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     constexpr int kRingCol0 = (kZopCols <= 32) ? 32 : 64;            // first column of the accumulator ring
     constexpr int NBUF = (kGroupCols - kRingCol0) / kBufCols;        // 3 or 2
     constexpr int kR2BlockBytes = RPAD * 128;                        // RPAD rows x 64 experts
-    using Sel = Selector<KCAP, FILTER, kEpiThreads, kCandCap, 8>;
+    using Sel = Selector<KCAP, FILTER, kEpiThreads, kCandCap, 8, 8, !FILTER>;
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -360,10 +360,13 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
     int* zop_done = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 32);    // [tg]: warps that have written their operand
     int* released = reinterpret_cast<int*>(ctl + B_COUNT * 8 + 48);    // [group][slot]: warps that have read a buffer out
     STAT(long long* issue_clk = reinterpret_cast<long long*>(ctl + B_COUNT * 8 + 96);)   // [group][slot]: when the refill was issued
+    // [token group][token][expert range]: the k-th value each range's thread has reached for its token (see `exchange`)
+    float* tau_pub = reinterpret_cast<float*>(ctl + 1024);
     const uint32_t bar0 = smem_u32(bars);
     auto bar = [&](int i) { return bar0 + 8u * (uint32_t)i; };
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x < kEpiThreads) { tau_pub[2 * threadIdx.x] = -INFINITY; tau_pub[2 * threadIdx.x + 1] = -INFINITY; }
     const int blk = blockIdx.x / p.msplit, split = blockIdx.x % p.msplit;
     const int tok0 = blk * p.block_tokens;
     const int live_tokens = min(p.block_tokens, p.T - tok0);
@@ -643,8 +646,32 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
         };
         // ---- after the two chunks of a buffer: fold if some token of the warp could overflow on the next buffer
         // (the first two buffers of a sweep are folded wholesale: with a near-empty list almost everything gets in)
+        // The expert ranges of a CTA sweep the same tokens, and every range would pay the expensive start of a sweep on its
+        // own.  After a fold a thread publishes two values of its list (KCAP entries, sorted): the last one, and the
+        // one at position KCAP/es - 1.  Both give lower bounds for the token's final KCAP-th value: at least KCAP logits
+        // reach any range's last value, and at least KCAP/es logits in every range, KCAP in all, reach the smallest
+        // of the values at position KCAP/es - 1.  The larger bound, lowered by a hair so that an equal logit (which a
+        // smaller id could still win) is kept, becomes the floor of this thread's own collection.
+        float2* const tau_mine = reinterpret_cast<float2*>(tau_pub) + (tgi * 128 + row_in_tg) * es;
+        auto exchange = [&]() {
+            if constexpr (!FILTER) {
+                if (es > 1) {
+                    tau_mine[esi] = make_float2(S.L.tau(), es == 4 ? S.L.v[KCAP / 4 - 1] : S.L.v[KCAP / 2 - 1]);
+                    float2 b = tau_mine[0];
+                    for (int e = 1; e < es; ++e) {
+                        const float2 o = tau_mine[e];
+                        b.x = fmaxf(b.x, o.x);
+                        b.y = fminf(b.y, o.y);
+                    }
+                    const float best = fmaxf(b.x, b.y);
+                    S.ext = fmaf(-fabsf(best), 2.4e-7f, best) - 1e-37f;       // strictly below `best` (-inf stays -inf)
+                    S.thr = fmaxf(S.thr, S.ext);
+                }
+            }
+        };
         auto fold_check = [&](int n) {
-            if (__any_sync(kFullMask, S.ptr >= S.warn)) {
+            const bool folds = __any_sync(kFullMask, S.ptr >= S.warn);
+            if (folds) {
                 STAT(st_fold++; const long long tr0 = clock64();)
                 if constexpr (FILTER) {
                     S.fold();
@@ -654,6 +681,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                 }
                 STAT(st_tfold += clock64() - tr0;)
             }
+            if (folds) exchange();
         };
 
         // ---- the sweep: buffer n of the group lives in ring slot n % NBUF.  A warp's loop is a chain of long

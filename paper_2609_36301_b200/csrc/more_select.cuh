@@ -118,7 +118,7 @@ __device__ __forceinline__ float bf_hi(uint32_t u) { return __uint_as_float(u & 
 // FILTER: the logits are approximate to within E; thr sits W = 2E below the list's last value, elements that land in
 // that zone (directly, or pushed out of the list) are kept in a second small per-token store, pruned when it fills
 // up; a token whose zone still overflows is flagged for the fallback.
-template <int KCAP, bool FILTER, int NT, int CAP, int PER_CHECK, int ZCAP = 8>
+template <int KCAP, bool FILTER, int NT, int CAP, int PER_CHECK, int ZCAP = 8, bool EXT = false>
 struct Selector {
     static constexpr int kCandValStride = NT * 16;   // bytes between successive value slots of one thread
     static constexpr int kCandColStride = NT * 4;    // ... and between its column slots
@@ -131,6 +131,7 @@ struct Selector {
     TopList<KCAP> L;
     float thr;
     float W;
+    float ext;        // EXT: a lower bound on the final k-th value known from elsewhere (strictly below it)
     uint32_t ptr, cptr, base, cbase, warn;
     uint32_t zptr, zbase;
     bool overflow;
@@ -139,6 +140,7 @@ struct Selector {
     {
         L.init();
         thr = -INFINITY;
+        ext = -INFINITY;
         W = w;
         base = ptr = first_val_slot;
         cbase = cptr = first_col_slot;
@@ -146,7 +148,7 @@ struct Selector {
         zbase = zptr = first_zone_slot;
         overflow = false;
     }
-    __device__ __forceinline__ float limit() const { return FILTER ? L.tau() - W : L.tau(); }
+    __device__ __forceinline__ float limit() const { return FILTER ? L.tau() - W : (EXT ? fmaxf(L.tau(), ext) : L.tau()); }
 
     // Drop the zone entries that have fallen more than W below the list; flag the token if the zone is still full.
     __device__ __forceinline__ void prune()
