@@ -292,7 +292,9 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
                 // a sweep starts with an empty list, so nearly every early logit is a candidate: worth ~160 chunks on a
                 // long range, about ten times its own length on a short one
                 const double range_chunks = 4.0 * ((blocks64 + es * s - 1) / (es * s));     // whole 64-expert steps
-                const double chunks = range_chunks + (range_chunks < 16.0 ? 10.0 * range_chunks : 160.0);
+                // (the expert ranges of a CTA share their thresholds, so together they pay one start, not es)
+                const double all_chunks = range_chunks * es;
+                const double chunks = range_chunks + (all_chunks < 16.0 ? 10.0 * all_chunks : 160.0) / es;
                 // warps per scheduler: one per group, except that a block of at most 64 tokens is spread over the
                 // lane quarters, one or two quarters per expert range (credited only to small problems: on long
                 // sweeps the latency term of this model is too optimistic for two warps per scheduler)
@@ -302,7 +304,7 @@ void plan_lowrank(int T, int h, int r, int M, int k, bool want_lse, int msplit, 
                 const double ktile = bt * 128.0 / 23.0 > 300.0 ? bt * 128.0 / 23.0 : 300.0;
                 double t = 9000.0 + ((h + 63) / 64) * ktile + chunks * per_chunk;
                 if (es > 1) t += 1500.0;
-                if (s > 1) t += 7000.0 + 60.0 * s + 1.5 * s * bt;      // park, last arriver, its merge of s lists per token
+                if (s > 1) t += 7000.0 + 30.0 * s + 0.75 * s * bt;     // park, last arriver, its merge of s lists per token
                 const double cost = waves * t;
                 if (cost < best * 0.999) {
                     best = cost;
