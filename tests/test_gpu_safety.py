@@ -111,3 +111,45 @@ def test_host_entry_point_from_two_threads_with_different_sizes():
     t1.start(); t2.start(); t1.join(); t2.join()
     assert not errors, errors
     assert mr.more_route_status() == 0
+
+
+def test_a_call_that_fails_on_the_host_touches_no_output():
+    """Every error the host can detect is detected before anything is enqueued: the outputs, out_counts included (which
+    a successful call clears first), keep what they held.  Misaligned operand, a shape the forced tensor-core path
+    cannot take, an expert split out of range, an unknown gate mode."""
+    import torch
+    T, h, r, M, k = 512, 256, 32, 1024, 8
+    case = inputs.gaussian_case(T, h, r, M, k, 0, seed=5)
+    X, R1, R2 = to_device(case)
+    idx = torch.full((T, k), -3, dtype=torch.int32, device="cuda")
+    gate = torch.full((T, k), -1.0, dtype=torch.float32, device="cuda")
+    counts = torch.full((M,), 77, dtype=torch.int32, device="cuda")
+
+    def untouched():
+        torch.cuda.synchronize()
+        return bool((idx == -3).all() and (gate == -1.0).all() and (counts == 77).all())
+
+    # (1) X one bf16 element off a 16-byte boundary
+    Xbig = torch.zeros((T * h + 8,), dtype=torch.bfloat16, device="cuda")
+    Xoff = Xbig[1:1 + T * h].view(T, h)
+    with pytest.raises(mr.MoreRouteError) as e:
+        mr.more_route_ex(Xoff, R1, R2, k, 0, idx, gate, counts)
+    assert e.value.code == -3 and untouched()          # MORE_ERR_ALIGN
+    # (2) a rank the tensor-core path cannot take, with that path forced
+    R1b = torch.zeros((h, 72), dtype=torch.bfloat16, device="cuda")
+    R2b = torch.zeros((72, M), dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(mr.MoreRouteError) as e:
+        mr.more_route_ex(X, R1b, R2b, k, 0, idx, gate, counts, path=mr.PATH_TCGEN05)
+    assert e.value.code == -2 and untouched()          # MORE_ERR_SHAPE
+    # (3) an expert split beyond the limit
+    with pytest.raises(mr.MoreRouteError) as e:
+        mr.more_route_ex(X, R1, R2, k, 0, idx, gate, counts, msplit=65)
+    assert e.value.code == -2 and untouched()
+    # (4) an unknown gate mode
+    with pytest.raises(mr.MoreRouteError) as e:
+        mr.more_route_ex(X, R1, R2, k, 7, idx, gate, counts)
+    assert e.value.code == -4 and untouched()          # MORE_ERR_MODE
+    # and the same buffers still work
+    mr.more_route_ex(X, R1, R2, k, 0, idx, gate, counts)
+    torch.cuda.synchronize()
+    assert mr.more_route_status() == 0 and int(counts.sum()) == T * k
