@@ -89,7 +89,10 @@ constexpr int kMaxStages1 = 8;                     // k-tiles of the projection 
 constexpr int kFallbackSlots = 16;                 // tokens re-routed per round of the fallback (one per epilogue warp)
 constexpr float kLog2e = 1.4426950408889634f;
 
-enum { kModeExact = 0, kModeExactLse = 1, kModeFilter = 2 };
+// (the ...Fan modes are the exact modes with the fanned-out merge of parked lists compiled in for lists longer than 8
+// entries: launched only when a token block is split over 8 or more CTAs, because that code costs the sweep of such
+// kernels ~3 %; lists of up to 8 entries always have it)
+enum { kModeExact = 0, kModeExactLse = 1, kModeFilter = 2, kModeExactFan = 3, kModeExactLseFan = 4 };
 
 struct RouteParams {
     int T, h, r, M, k, gate_mode;
@@ -153,7 +156,7 @@ __device__ __forceinline__ void write_token(const RouteParams& p, int64_t row, c
 // scratch: on return the thread of every live token (`writer`, row `row_in_blk` of the block) holds the token's
 // list and (m, Z) pair.  Called by all 512 epilogue threads; the ring (idle by then) is working space.  A function
 // of its own so that its register needs stay out of the sweep's allocation.
-template <int KCAP, bool LSE>
+template <int KCAP, bool LSE, bool FAN>
 __device__ __forceinline__ void merge_parked_lists(const RouteParams& p, int blk, int etid, int live_tokens, uint8_t* ring_ptr,
                                                 int row_in_blk, bool writer, TopList<KCAP>& G, float& gm, float& gz)
 {
@@ -205,14 +208,15 @@ __device__ __forceinline__ void merge_parked_lists(const RouteParams& p, int blk
     // With few tokens and many splits (decode shapes) one thread per token would walk all lists one
     // L2 round trip after the other; instead `fan` threads per token merge a contiguous share of the
     // ranges each, park their result in the idle ring, and the token's own thread merges those.
-    // (Lists of up to 8 entries only: with longer ones this code raises the register needs of the whole kernel, which
-    // costs the sweep of the large k = 16 configurations more than it gains here.)
+    // (FAN: always for lists of up to 8 entries; for longer ones this code raises the register needs of the whole kernel,
+    // which costs the sweep of the large k = 16 configurations ~3 %, so it is compiled into instantiations of their own
+    // that are launched only when a token block is split over 8 or more CTAs.)
     int fan = 1;
-    if constexpr (KCAP <= 8)
+    if constexpr (FAN)
         while (fan < 16 && 2 * fan * p.block_tokens <= kEpiThreads && 4 * fan <= p.msplit) fan *= 2;
     if (fan == 1) {
         if (writer) merge_range(G, gm, gz, row_in_blk, 0, p.msplit);
-    } else if constexpr (KCAP <= 8) {
+    } else if constexpr (FAN) {
         // The lists are first copied into the idle ring with coalesced, independent loads (one L2
         // round trip for all of them instead of one per list and thread), in batches of `lb` lists per
         // token when they do not fit at once; a token's rows are skewed by 16 bytes against the banks.
@@ -221,7 +225,7 @@ __device__ __forceinline__ void merge_parked_lists(const RouteParams& p, int blk
         // in log2(fan) levels.
         const int bt = p.block_tokens;
         constexpr int kPerList = KCAP * 8 + 8;
-    constexpr int kInFlight = 4;                          // loads per array and thread in flight during the copy
+    constexpr int kInFlight = KCAP <= 8 ? 4 : 2;          // loads per array and thread in flight during the copy
         float* sv = reinterpret_cast<float*>(ring_ptr);                  // [fan][KCAP][bt]
         int* si = reinterpret_cast<int*>(sv + fan * KCAP * bt);         // [fan][KCAP][bt]
         float2* smz = reinterpret_cast<float2*>(si + fan * KCAP * bt);  // [fan][bt]
@@ -335,7 +339,8 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                      const __grid_constant__ CUtensorMap map_r2, const RouteParams p)
 {
     constexpr bool FILTER = MODE == kModeFilter;
-    constexpr bool LSE = MODE == kModeExactLse;
+    constexpr bool LSE = MODE == kModeExactLse || MODE == kModeExactLseFan;
+    constexpr bool FAN = KCAP <= 8 || MODE == kModeExactFan || MODE == kModeExactLseFan;
     constexpr int kKSteps = RPAD / 16;                               // UMMA K = 16
     constexpr int kMmasPerBuf = FILTER ? kKSteps : 2 * kKSteps;      // exact modes: hi then lo into one accumulator
     constexpr int kZopCols = FILTER ? RPAD / 2 : RPAD;               // A operand: two bf16 per 32-bit column
@@ -1003,7 +1008,7 @@ route_lowrank_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_con
                     __threadfence();
                     TopList<KCAP> G;
                     float gm, gz;
-                    merge_parked_lists<KCAP, LSE>(p, blk, etid, live_tokens, ring_ptr, row_in_blk, writer, G, gm, gz);
+                    merge_parked_lists<KCAP, LSE, FAN>(p, blk, etid, live_tokens, ring_ptr, row_in_blk, writer, G, gm, gz);
                     hist_clear();
                     if (writer) write_token<KCAP>(p, row, G, gm, gz, hist);
                     hist_flush();
@@ -1131,6 +1136,12 @@ KernelFn kernel_mode(int mode)
     switch (mode) {
         case kModeExact: return kernel_ready<RPAD, KCAP, kModeExact>();
         case kModeExactLse: return kernel_ready<RPAD, KCAP, kModeExactLse>();
+        case kModeExactFan:
+            if constexpr (KCAP > 8) return kernel_ready<RPAD, KCAP, kModeExactFan>();
+            return kernel_ready<RPAD, KCAP, kModeExact>();
+        case kModeExactLseFan:
+            if constexpr (KCAP > 8) return kernel_ready<RPAD, KCAP, kModeExactLseFan>();
+            return kernel_ready<RPAD, KCAP, kModeExactLse>();
         default:
 #ifdef MORE_WITH_FILTER
             if constexpr (KCAP <= 16) return kernel_ready<RPAD, KCAP, kModeFilter>();
@@ -1254,6 +1265,7 @@ int launch_lowrank(const RouteArgs& a, DeviceCtx& ctx, const Plan& p, void* scra
     }
     const bool lse = (a.gate_mode == MORE_GATE_FULL_SOFTMAX) || (a.out_lse != nullptr);
     int mode = lse ? kModeExactLse : kModeExact;
+    if (p.msplit >= 8) mode = lse ? kModeExactLseFan : kModeExactFan;
     if (p.filter) {
         if (lse || a.k > 16) return MORE_ERR_SHAPE;
         mode = kModeFilter;
